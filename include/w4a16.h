@@ -1,0 +1,147 @@
+/*
+ * w4a16.h -- C ABI of the B200 (sm_100a) W4A16 matrix multiplication library.
+ *
+ *     C[M,N] = A[M,K] . Dequant(W)[K,N],   Dequant(W) = s (W - z)        (paper Eq. 2)
+ *
+ * A is FP16, W is unsigned INT4 (0..15) with one FP16 scale s and one integer zero
+ * point z (0..15) per group of `group` = 128 consecutive k and per column n,
+ * accumulation is FP32 and C is FP16 (Algorithm 1: dequantize, Split-K multiply,
+ * reduce + FP32->FP16 cast).
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a parameter says
+ *     "host".  The library allocates no device memory, keeps no reference to a buffer
+ *     after the work it enqueued has completed, and never frees anything.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream) and return without waiting.  Argument errors are detected on the
+ *     host, returned at once, and launch nothing.
+ *   - Return value: W4A16_OK (0) or a negative W4A16_ERR_* code; w4a16_strerror()
+ *     names it.  Nothing is printed, nothing throws, nothing exits.
+ *   - FP16 values cross the boundary as their 16-bit patterns (uint16_t).
+ *   - Device code exists for sm_100a only; on any other device the launching calls
+ *     return W4A16_ERR_ARCH.
+ *
+ * Raw layout (what w4a16_pack consumes; Section 2.2: "4-bit values must be packed into
+ * larger data types such as INT32"):
+ *   Wq_raw  uint32 [K/8, N] row-major; bits 4i..4i+3 of Wq_raw[kk, n] hold q[8 kk + i, n]
+ *   S_raw   FP16   [K/group, N] row-major
+ *   Z_raw   uint8  [K/group, N] row-major, one zero point (0..15) per byte
+ * Packed layout (what the kernels consume): opaque; sizes from w4a16_packed_*_bytes.
+ *
+ * Preconditions shared by pack / dequant / gemm:  group == 128, K > 0, K % 128 == 0,
+ * N > 0, N % 64 == 0; all buffers 16-byte aligned.  Violations -> W4A16_ERR_SHAPE /
+ * W4A16_ERR_ALIGN / W4A16_ERR_NULL.
+ */
+#ifndef W4A16_H_
+#define W4A16_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *w4a16_stream_t; /* a cudaStream_t; NULL = default stream */
+
+enum {
+    W4A16_OK = 0,
+    W4A16_ERR_NULL = -1,          /* a required pointer is NULL */
+    W4A16_ERR_SHAPE = -2,         /* M, N, K or group outside the supported set */
+    W4A16_ERR_ALIGN = -3,         /* a buffer is not 16-byte aligned */
+    W4A16_ERR_SPLITK = -4,        /* split_k < 0 or > K/group */
+    W4A16_ERR_WORKSPACE = -5,     /* split_k > 1 needs more workspace than was set */
+    W4A16_ERR_CUDA = -6,          /* a CUDA runtime call failed (launch, attribute, copy) */
+    W4A16_ERR_ARCH = -7,          /* current device is not sm_100 */
+    W4A16_ERR_DEVICE_STATUS = -8, /* a kernel gave up on a bounded wait; see w4a16_device_status */
+    W4A16_ERR_PATH = -9           /* requested kernel path cannot run this shape */
+};
+
+/* Kernel selection for w4a16_gemm_ex.  AUTO picks by shape. */
+enum {
+    W4A16_PATH_AUTO = 0,
+    W4A16_PATH_SIMPLE = 1, /* plain FP32-FMA kernel, any M; two-kernel Split-K reduce */
+    W4A16_PATH_DECODE = 2, /* small-M bandwidth-bound kernel (M <= 64): TMA bulk staging,
+                              in-register unpack, warp-level tensor-core MMA */
+    W4A16_PATH_TILE = 3    /* tcgen05 / TMEM tile kernel for large M */
+};
+
+const char *w4a16_strerror(int code);
+
+/* Sizes in bytes of the three packed buffers for a [K, N] weight matrix (0 if the shape
+ * is not supported).  The packed form holds exactly the information of the raw form:
+ * K*N/2 bytes of nibbles, 2 bytes per scale, 4 bits per zero point. */
+size_t w4a16_packed_wq_bytes(int N, int K, int group);
+size_t w4a16_packed_s_bytes(int N, int K, int group);
+size_t w4a16_packed_z_bytes(int N, int K, int group);
+
+/* Split-K (Algorithm 1, Phase 2/3) keeps FP32 partial results C_i in a caller-owned
+ * device workspace.  w4a16_workspace_bytes: bytes needed by w4a16_gemm for this shape
+ * and split_k (split_k == 0 means "whatever w4a16_choose_split_k picks"); 0 when no
+ * workspace is needed.
+ * w4a16_set_workspace: registers the buffer for the CURRENT device (one per device, per
+ * process; replaces the previous one; dev_ptr == NULL, bytes == 0 unregisters).  The
+ * buffer must be 256-byte aligned, stays owned by the caller and must outlive every gemm
+ * call enqueued while it is registered.  The call zeroes the buffer's first 4 KiB on the
+ * default stream and waits for that.  gemm calls that need the workspace and overlap on
+ * the GPU (different streams) race on it; serialise them or use split_k = 1. */
+size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k);
+int w4a16_set_workspace(void *dev_ptr, size_t bytes);
+
+/* The split factor S the library picks for a shape when split_k == 0 (the paper takes S
+ * as an input and gives no rule; Section 4.1 says when it pays: K >> N).  Always a value
+ * w4a16_gemm accepts; >= 1.  `path` as in w4a16_gemm_ex. */
+int w4a16_choose_split_k(int M, int N, int K, int group);
+int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path);
+
+/* Offline reorder of the raw nibbles, scales and zero points into the packed layout
+ * (pure data movement, a bijection; Section 2.2 storage packing).  Reads the three raw
+ * device arrays, writes the three packed device buffers (sizes above). */
+int w4a16_pack(const uint32_t *Wq_raw, const uint16_t *S_raw, const uint8_t *Z_raw,
+               void *Wq, void *S, void *Z, int N, int K, int group, w4a16_stream_t stream);
+
+/* Algorithm 1, Phase 1 as a standalone operation: W16[k, n] = fp16_rn((q - z) * s),
+ * one rounding to nearest-even, subnormals kept.  Wq, S, Z are PACKED buffers.
+ * W16: FP16 [K, N] row-major, fully overwritten. */
+int w4a16_dequant(const void *Wq, const void *S, const void *Z, uint16_t *W16,
+                  int N, int K, int group, w4a16_stream_t stream);
+
+/* Eq. 2 / Algorithm 1: C = A . Dequant(W), FP32 accumulation, Split-K over `split_k`
+ * slices of whole groups (slice sizes differ by at most one group, the first
+ * (K/group) mod split_k slices get the extra one), partial results summed in ascending
+ * slice order in FP32, one FP32->FP16 rounding (nearest-even) at the end.
+ *   A   FP16 [M, K] row-major (K contiguous), M >= 1
+ *   Wq, S, Z   packed buffers from w4a16_pack
+ *   C   FP16 [M, N] row-major, fully overwritten (no beta)
+ *   split_k   0 = automatic, else 1 <= split_k <= K/group (some paths cap it lower and
+ *             return W4A16_ERR_SPLITK beyond their cap)
+ * Results are bit-identical from run to run for fixed arguments.  If the chosen
+ * split needs workspace and too little is registered: W4A16_ERR_WORKSPACE. */
+int w4a16_gemm(const uint16_t *A, const void *Wq, const void *S, const void *Z, uint16_t *C,
+               int M, int N, int K, int group, int split_k, w4a16_stream_t stream);
+
+/* Same operation with the kernel path forced (W4A16_PATH_*); for tests and benchmarks.
+ * W4A16_ERR_PATH if that path does not support the shape. */
+int w4a16_gemm_ex(const uint16_t *A, const void *Wq, const void *S, const void *Z, uint16_t *C,
+                  int M, int N, int K, int group, int split_k, int path, w4a16_stream_t stream);
+
+/* End-to-end form of w4a16_gemm for callers whose activations live in HOST memory:
+ * copies A_host (FP16 [M, K], ideally pinned) into the caller's device staging buffer
+ * A_dev, runs w4a16_gemm into the device staging buffer C_dev, and copies the result
+ * into C_host (FP16 [M, N]); all three steps are enqueued on `stream` in order.  The
+ * host buffers must stay valid until the stream has run them.  Weights stay resident
+ * on the device (they are the model's parameters, packed once). */
+int w4a16_gemm_host(const uint16_t *A_host, uint16_t *A_dev, const void *Wq, const void *S,
+                    const void *Z, uint16_t *C_dev, uint16_t *C_host, int M, int N, int K,
+                    int group, int split_k, w4a16_stream_t stream);
+
+/* Kernels never wait without a limit: a wait that runs out records a code in a status
+ * word on the device and the kernel returns.  This call synchronises the current
+ * device, copies the word to *status_out (0 = no kernel ever gave up) and clears it.
+ * Returns W4A16_ERR_DEVICE_STATUS if it was nonzero. */
+int w4a16_device_status(int *status_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W4A16_H_ */

@@ -30,6 +30,7 @@
 #include <stddef.h>
 #include <string.h>
 #include <math.h>
+#include <stdlib.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -130,23 +131,40 @@ void orc_dequant(const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
 /* ---- C = A . Dequant(W) in FP64 (Eq. 2) ---- */
 
 /* A: FP16 bits [M, K] row-major.  C_ref: double [M, N] row-major.
- * Columns n0 <= n < n1 only are written (n0 = 0, n1 = N for everything). */
-void orc_gemm_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
-                   int M, int N, int K, int group, int n0, int n1, double *C_ref)
+ * Only columns n0 <= n < n1 are written, and only k0 <= k < k1 is summed
+ * (n0 = 0, n1 = N, k0 = 0, k1 = K for the whole product).  Column n of
+ * Dequant(W) is formed once (FP16-rounded, then widened) and every row of A is
+ * multiplied into it. */
+void orc_gemm_kslice_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                          int M, int N, int K, int group, int k0, int k1, int n0, int n1,
+                          double *C_ref)
 {
-    #pragma omp parallel for schedule(static)
-    for (int n = n0; n < n1; ++n) {
-        for (int m = 0; m < M; ++m) {
-            double acc = 0.0;
-            for (int k = 0; k < K; ++k) {
+    #pragma omp parallel
+    {
+        double *wcol = (double *)malloc(sizeof(double) * (size_t)K);
+        #pragma omp for schedule(static)
+        for (int n = n0; n < n1; ++n) {
+            for (int k = k0; k < k1; ++k) {
                 int g = k / group;
                 uint16_t w16 = orc_dequant_one(orc_q_at(Wq, N, k, n),
                                                Z[(size_t)g * N + n], S[(size_t)g * N + n]);
-                acc += (double)orc_f16_to_f32(A[(size_t)m * K + k]) * (double)orc_f16_to_f32(w16);
+                wcol[k] = (double)orc_f16_to_f32(w16);
             }
-            C_ref[(size_t)m * N + n] = acc;
+            for (int m = 0; m < M; ++m) {
+                double acc = 0.0;
+                for (int k = k0; k < k1; ++k)
+                    acc += (double)orc_f16_to_f32(A[(size_t)m * K + k]) * wcol[k];
+                C_ref[(size_t)m * N + n] = acc;
+            }
         }
+        free(wcol);
     }
+}
+
+void orc_gemm_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                   int M, int N, int K, int group, int n0, int n1, double *C_ref)
+{
+    orc_gemm_kslice_cols(A, Wq, S, Z, M, N, K, group, 0, K, n0, n1, C_ref);
 }
 
 void orc_gemm(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
@@ -159,19 +177,7 @@ void orc_gemm(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const ui
 void orc_gemm_kslice(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
                      int M, int N, int K, int group, int k0, int k1, double *C_part)
 {
-    #pragma omp parallel for schedule(static)
-    for (int n = 0; n < N; ++n) {
-        for (int m = 0; m < M; ++m) {
-            double acc = 0.0;
-            for (int k = k0; k < k1; ++k) {
-                int g = k / group;
-                uint16_t w16 = orc_dequant_one(orc_q_at(Wq, N, k, n),
-                                               Z[(size_t)g * N + n], S[(size_t)g * N + n]);
-                acc += (double)orc_f16_to_f32(A[(size_t)m * K + k]) * (double)orc_f16_to_f32(w16);
-            }
-            C_part[(size_t)m * N + n] = acc;
-        }
-    }
+    orc_gemm_kslice_cols(A, Wq, S, Z, M, N, K, group, k0, k1, 0, N, C_part);
 }
 
 /* ---- exact case: integer A, power-of-two scales ----

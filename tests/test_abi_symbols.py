@@ -1,0 +1,89 @@
+"""The C-ABI library loads, exports every symbol include/w4a16.h declares, and validates
+arguments on the host before touching a device (no compute calls here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2601_16536_b200 import binding as B
+from paper_2601_16536_b200 import build as libbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    libbuild.build_library()
+    return B.load()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "w4a16.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(w4a16_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(B.EXPORTS)
+
+
+def test_packed_sizes_hold_exactly_the_raw_information(lib):
+    for N, K in [(64, 128), (4096, 4096), (4096, 11008), (8192, 28672), (22016, 4096)]:
+        assert lib.w4a16_packed_wq_bytes(N, K, 128) == K * N // 2
+        assert lib.w4a16_packed_s_bytes(N, K, 128) == (K // 128) * N * 2
+        assert lib.w4a16_packed_z_bytes(N, K, 128) == (K // 128) * N // 2
+    # unsupported shapes report size 0
+    assert lib.w4a16_packed_wq_bytes(100, 4096, 128) == 0
+    assert lib.w4a16_packed_wq_bytes(4096, 4000, 128) == 0
+    assert lib.w4a16_packed_wq_bytes(4096, 4096, 64) == 0
+
+
+def test_choose_split_k_is_always_acceptable(lib):
+    for M in (1, 2, 4, 8, 16, 32, 64, 256, 1024, 4096):
+        for N, K in [(4096, 4096), (4096, 11008), (8192, 28672), (12288, 4096), (22016, 4096),
+                     (8192, 8192), (64, 128), (64, 256)]:
+            s = lib.w4a16_choose_split_k(M, N, K, 128)
+            assert 1 <= s <= K // 128
+            for path in (1, 2, 3):
+                s = lib.w4a16_choose_split_k_ex(M, N, K, 128, path)
+                assert 1 <= s <= K // 128
+            ws = lib.w4a16_workspace_bytes(M, N, K, 128, 0)
+            assert ws == lib.w4a16_workspace_bytes(M, N, K, 128, lib.w4a16_choose_split_k(M, N, K, 128))
+    assert lib.w4a16_workspace_bytes(4, 4096, 4096, 128, 1) == 0
+    assert lib.w4a16_workspace_bytes(4, 4096, 4096, 128, 4) >= 4 * 4 * 4096 * 4
+
+
+def test_argument_errors_are_reported_before_any_device_work(lib):
+    buf = (ctypes.c_uint8 * 4096)()
+    p = ctypes.addressof(buf)
+    p = (p + 15) // 16 * 16
+    assert lib.w4a16_gemm(None, p, p, p, p, 1, 64, 128, 128, 1, None) == -1
+    assert lib.w4a16_gemm(p, p, p, p, None, 1, 64, 128, 128, 1, None) == -1
+    assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 128, 64, 1, None) == -2      # group
+    assert lib.w4a16_gemm(p, p, p, p, p, 1, 60, 128, 128, 1, None) == -2     # N % 64
+    assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 100, 128, 1, None) == -2     # K % 128
+    assert lib.w4a16_gemm(p, p, p, p, p, 0, 64, 128, 128, 1, None) == -2     # M
+    assert lib.w4a16_gemm(p + 2, p, p, p, p, 1, 64, 128, 128, 1, None) == -3  # alignment
+    assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 128, 128, 2, None) == -4     # split_k > K/group
+    assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 128, 128, -1, None) == -4
+    assert lib.w4a16_gemm_ex(p, p, p, p, p, 1, 64, 128, 128, 1, 9, None) == -9
+    assert lib.w4a16_pack(None, p, p, p, p, p, 64, 128, 128, None) == -1
+    assert lib.w4a16_pack(p, p, p, p, p, p, 64, 128, 32, None) == -2
+    assert lib.w4a16_dequant(p, p, p, None, 64, 128, 128, None) == -1
+    assert lib.w4a16_dequant(p, p, p, p + 4, 64, 128, 128, None) == -3
+    assert lib.w4a16_gemm_host(None, p, p, p, p, p, p, 1, 64, 128, 128, 1, None) == -1
+    assert lib.w4a16_device_status(None) == -1
+    for code in range(-9, 1):
+        assert len(B.strerror(code)) > 1
+
+
+def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        B.load()

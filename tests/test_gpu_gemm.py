@@ -1,0 +1,141 @@
+"""GPU parity of w4a16_gemm against the FP64 oracle (Eq. 2; Algorithm 1 Split-K), through the C ABI.
+
+Tolerances (stated by the benchmark spec): relative Frobenius error <= 1e-3 and per element
+|dC| <= 2e-3 (1 + |C_ref|).  With exactly representable inputs the result is unique and must be
+bit-equal for every path and split.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_16536_b200 import binding as B
+from paper_2601_16536_b200 import workloads as wl
+from gpu_util import assert_close, c_bits, c_f64, ensure_ws, pack_problem, to_dev
+
+pytestmark = pytest.mark.gpu
+
+PATHS = {"simple": B.PATH_SIMPLE, "decode": B.PATH_DECODE}
+
+
+def _run(d, M, N, K, split_k, path):
+    pw = pack_problem(d, N, K)
+    ws = ensure_ws(M, N, K, split_k if split_k else B.w4a16_choose_split_k(M, N, K, 128, path))
+    C = B.w4a16_gemm(to_dev(d["A"]), pw, split_k=split_k, path=path)
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    del ws
+    return C
+
+
+# several 64-column tiles, ragged group counts (5, 7, 9 groups: not a multiple of the 4 groups a
+# stage holds, nor of the splits), every batch-block edge
+SMALL = [(1, 128, 64), (1, 640, 192), (3, 896, 128), (8, 1152, 256), (9, 640, 128),
+         (16, 1152, 192), (5, 4096, 512)]
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("M,K,N", SMALL)
+@pytest.mark.parametrize("split_k", [1, 2, 3])
+def test_small_shapes_match_oracle(path, M, K, N, split_k):
+    if split_k > K // 128:
+        pytest.skip("more splits than groups")
+    d = wl.make_problem(M, K, N, seed=M * 1000 + K + N)
+    C = _run(d, M, N, K, split_k, PATHS[path])
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+    assert_close(c_f64(C), ref, "%s M%d K%d N%d S%d" % (path, M, K, N, split_k))
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("M", [17, 33, 64])
+def test_batch_larger_than_one_block(path, M):
+    K, N = 768, 128
+    d = wl.make_problem(M, K, N, seed=M)
+    C = _run(d, M, N, K, 2, PATHS[path])
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+    assert_close(c_f64(C), ref, "%s M%d" % (path, M))
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+def test_exact_inputs_are_bit_equal_for_every_split(path):
+    # A in {-1,0,1}, s = 2^e: every partial sum is exact in FP32 in any order, so the FP16
+    # result is unique (closed form) -- any split, any path must return exactly it
+    M, K, N = 7, 2304, 192    # 18 groups
+    d = wl.make_exact_problem(M, K, N, seed=90)
+    want = oracle.gemm_int(d["A_int"], d["Wq"], d["E"], d["Z"], M, N, K, 128)
+    for split_k in (1, 2, 4, 5, 8, 16, 18):
+        C = _run(d, M, N, K, split_k, PATHS[path])
+        assert np.array_equal(c_bits(C), want), "split_k=%d" % split_k
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+def test_q_equals_z_gives_zero_and_scaling_is_linear(path):
+    M, K, N = 4, 512, 128
+    d = wl.make_problem(M, K, N, seed=91)
+    dz = dict(d)
+    dz["Wq"] = np.repeat(d["Z"].astype(np.uint32) * np.uint32(0x11111111), 16, axis=0)
+    C0 = _run(dz, M, N, K, 1, PATHS[path])
+    assert np.all(c_f64(C0) == 0.0)
+    d2 = dict(d)
+    d2["S"] = (d["S"].view(np.float16) * np.float16(2)).view(np.uint16)
+    C1 = c_f64(_run(d, M, N, K, 1, PATHS[path]))
+    C2 = c_f64(_run(d2, M, N, K, 1, PATHS[path]))
+    assert np.array_equal(C2, 2.0 * C1)   # power-of-two scaling commutes with every rounding
+
+
+def test_results_are_bit_identical_run_to_run():
+    M, K, N = 16, 11008, 512
+    d = wl.make_problem(M, K, N, seed=92)
+    pw = pack_problem(d, N, K)
+    A = to_dev(d["A"])
+    ws = ensure_ws(M, N, K, 16)
+    for split_k in (1, 4, 16):
+        first = c_bits(B.w4a16_gemm(A, pw, split_k=split_k, path=B.PATH_DECODE))
+        for _ in range(5):
+            again = c_bits(B.w4a16_gemm(A, pw, split_k=split_k, path=B.PATH_DECODE))
+            assert np.array_equal(first, again)
+    del ws
+
+
+def test_auto_path_and_split_match_oracle():
+    for M, K, N in [(1, 4096, 4096), (4, 11008, 1024), (16, 2048, 2048)]:
+        d = wl.make_problem(M, K, N, seed=93 + M)
+        C = _run(d, M, N, K, 0, B.PATH_AUTO)
+        ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+        assert_close(c_f64(C), ref, "auto M%d K%d N%d" % (M, K, N))
+
+
+def test_workspace_errors():
+    M, K, N = 4, 1024, 128
+    d = wl.make_problem(M, K, N, seed=94)
+    pw = pack_problem(d, N, K)
+    A = to_dev(d["A"])
+    B.w4a16_set_workspace(None)
+    with pytest.raises(B.W4A16Error) as e:
+        B.w4a16_gemm(A, pw, split_k=4, path=B.PATH_DECODE)
+    assert e.value.code == -5
+    small = torch.empty(8192, dtype=torch.uint8, device="cuda")
+    B.w4a16_set_workspace(small[(-small.data_ptr()) % 256:][:4096 + 256])
+    with pytest.raises(B.W4A16Error) as e:
+        B.w4a16_gemm(A, pw, split_k=4, path=B.PATH_DECODE)
+    assert e.value.code == -5
+    B.w4a16_set_workspace(None)
+    # split_k = 1 needs none
+    B.w4a16_gemm(A, pw, split_k=1, path=B.PATH_DECODE)
+    torch.cuda.synchronize()
+
+
+def test_host_buffer_entry_point_matches_device_call():
+    M, K, N = 8, 1024, 256
+    d = wl.make_problem(M, K, N, seed=95)
+    pw = pack_problem(d, N, K)
+    ws = ensure_ws(M, N, K, 0)
+    A_host = torch.from_numpy(d["A"].view(np.float16)).pin_memory()
+    C_host = torch.empty((M, N), dtype=torch.float16).pin_memory()
+    A_dev = torch.empty((M, K), dtype=torch.float16, device="cuda")
+    C_dev = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    B.w4a16_gemm_host(A_host, A_dev, pw, C_dev, C_host)
+    torch.cuda.synchronize()
+    C = B.w4a16_gemm(to_dev(d["A"]), pw)
+    assert np.array_equal(C_host.numpy().view(np.uint16), c_bits(C))
+    del ws
