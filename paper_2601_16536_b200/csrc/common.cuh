@@ -147,4 +147,17 @@ __device__ __forceinline__ Frag4 unpack_word(uint32_t w, __half2 zlo, __half2 zh
     return f;
 }
 
+// One packed word -> four FP16 pairs of w16 = fp16_rn((q - z) * s): exact (q - z), then one
+// FP16 multiply by the row's scale (both halves of s_lo / s_hi hold the scale of n_lo / n_hi).
+// This is Algorithm 1's "Dequantize to FP16": the multiplicand of the GEMM is the FP16-rounded
+// weight, so every kernel that feeds tensor cores goes through here.
+__device__ __forceinline__ Frag4 dequant_word(uint32_t w, __half2 zlo, __half2 zhi, __half2 s_lo, __half2 s_hi) {
+    Frag4 f = unpack_word(w, zlo, zhi);
+    f.lo_a = __hmul2(f.lo_a, s_lo);
+    f.hi_a = __hmul2(f.hi_a, s_hi);
+    f.lo_b = __hmul2(f.lo_b, s_lo);
+    f.hi_b = __hmul2(f.hi_b, s_hi);
+    return f;
+}
+
 }  // namespace w4a16

@@ -4,11 +4,10 @@
 // warp streams the slice's packed blocks (16 KiB = 4 groups per stage, one TMA bulk copy)
 // and the matching activation rows into a multi-stage shared-memory ring guarded by
 // mbarriers.  Four consumer warps each take one group per stage: a 128-bit shared load
-// gives a lane the A-fragment nibbles of a 16-row sub-tile, two logic ops and one FP16
-// op per register turn them into exact (q - z), and an m16n8k16 tensor-core MMA with
-// the WEIGHTS as the 16-row operand (MMA rows = n, MMA columns = batch rows) accumulates
-// the group in FP32; the group's FP32 sums are then scaled by s (FP32) into the running
-// accumulators.  The four warps' partial sums (disjoint k) are added in warp order
+// gives a lane the A-fragment nibbles of a 16-row sub-tile, a logic op and two FP16 ops
+// per register turn them into w16 = fp16_rn((q - z) s), and an m16n8k16 tensor-core MMA
+// with the WEIGHTS as the 16-row operand (MMA rows = n, MMA columns = batch rows)
+// accumulates in FP32.  The four warps' partial sums (disjoint k) are added in warp order
 // through shared memory; the result goes to C (split_k == 1) or to the FP32 Split-K
 // workspace.
 #pragma once
@@ -142,13 +141,14 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
             const uint32_t zw = z_s[lg * kZBlockWords + gq];
             const uint32_t sw[4] = {sraw.x, sraw.y, sraw.z, sraw.w};
 
-            float tmp[4][MB][4];
+            __half2 s_lo[4], s_hi[4], zlo[4], zhi[4];
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) tmp[r][mb][i] = 0.f;
+            for (int r = 0; r < 4; ++r) {
+                s_lo[r] = __half2half2(__low2half(u32_as_h2(sw[r])));   // row 16r + gq
+                s_hi[r] = __half2half2(__high2half(u32_as_h2(sw[r])));  // row 16r + gq + 8
+                zlo[r] = u32_as_h2(zmagic_lo((zw >> (8 * r)) & 15u));
+                zhi[r] = u32_as_h2(zmagic_hi((zw >> (8 * r + 4)) & 15u));
+            }
 
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -169,27 +169,14 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
                 }
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
-                    const __half2 zlo = u32_as_h2(zmagic_lo((zw >> (8 * r)) & 15u));
-                    const __half2 zhi = u32_as_h2(zmagic_hi((zw >> (8 * r + 4)) & 15u));
                     const uint4 wv = wsm[(c * 4 + r) * 32 + lane];
                     const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const Frag4 f = unpack_word(ww[j], zlo, zhi);
+                        const Frag4 f = dequant_word(ww[j], zlo[r], zhi[r], s_lo[r], s_hi[r]);
 #pragma unroll
-                        for (int mb = 0; mb < MB; ++mb) mma_m16n8k16(tmp[r][mb], f, bw[mb][2 * j], bw[mb][2 * j + 1]);
+                        for (int mb = 0; mb < MB; ++mb) mma_m16n8k16(acc[r][mb], f, bw[mb][2 * j], bw[mb][2 * j + 1]);
                     }
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const float2 sf = __half22float2(u32_as_h2(sw[r]));  // (s of row 16r+gq, s of row 16r+gq+8)
-#pragma unroll
-                for (int mb = 0; mb < MB; ++mb) {
-                    acc[r][mb][0] = fmaf(sf.x, tmp[r][mb][0], acc[r][mb][0]);
-                    acc[r][mb][1] = fmaf(sf.x, tmp[r][mb][1], acc[r][mb][1]);
-                    acc[r][mb][2] = fmaf(sf.y, tmp[r][mb][2], acc[r][mb][2]);
-                    acc[r][mb][3] = fmaf(sf.y, tmp[r][mb][3], acc[r][mb][3]);
                 }
             }
         }

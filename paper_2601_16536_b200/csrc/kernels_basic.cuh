@@ -81,10 +81,8 @@ __global__ void dequant_kernel(const uint32_t* __restrict__ Wq, const __half* __
     __half s_lo = S[blk * kSBlockHalves + gq * 8 + r * 2];
     __half s_hi = S[blk * kSBlockHalves + gq * 8 + r * 2 + 1];
 
-    Frag4 f = unpack_word(Wq[idx], zlo, zhi);
-    __half2 sl = __half2half2(s_lo), sh = __half2half2(s_hi);
-    __half2 wa = __hmul2(f.lo_a, sl), wb = __hmul2(f.lo_b, sl);
-    __half2 wc = __hmul2(f.hi_a, sh), wd = __hmul2(f.hi_b, sh);
+    const Frag4 f = dequant_word(Wq[idx], zlo, zhi, __half2half2(s_lo), __half2half2(s_hi));
+    const __half2 wa = f.lo_a, wb = f.lo_b, wc = f.hi_a, wd = f.hi_b;
     __half* p = W16 + (size_t)k0 * N + n_lo;
     p[0] = __low2half(wa);
     p[(size_t)N] = __high2half(wa);
