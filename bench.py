@@ -179,17 +179,32 @@ class Layer:
         return pw
 
 
-def _time_calls(fn, n_warm, n_timed, torch):
-    for _ in range(n_warm):
+def _capture(fn, n, torch):
+    """A CUDA graph of n consecutive calls of fn (launches recorded once, replayed without
+    per-call host work, so the device time of back-to-back kernels is what gets measured)."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(n):
+            fn()
+    return g
+
+
+def _time_calls(fn, n_warm, n_timed, torch, per_graph=32):
+    """Seconds per call: `fn` captured per_graph times into a CUDA graph, replayed."""
+    for _ in range(max(3, n_warm)):
         fn()
+    torch.cuda.synchronize()
+    g = _capture(fn, per_graph, torch)
+    reps = max(1, n_timed // per_graph)
+    g.replay()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(n_timed):
-        fn()
+    for _ in range(reps):
+        g.replay()
     e1.record()
     torch.cuda.synchronize()
-    return e0.elapsed_time(e1) * 1e-3 / n_timed   # seconds per call
+    return e0.elapsed_time(e1) * 1e-3 / (reps * per_graph)
 
 
 def run_ours(args):
@@ -215,7 +230,7 @@ def run_ours(args):
     acts = [_to_dev(a, torch) for a in acts_np]
     outs = [torch.empty((M, N), dtype=torch.float16, device="cuda") for M in SWEEP_M]
     splits = [args.split_k if args.split_k else B.w4a16_choose_split_k(M, N, K) for M in SWEEP_M]
-    ws_need = max([B.w4a16_workspace_bytes(M, N, K, 128, s) for M, s in zip(SWEEP_M, splits)] + [4096])
+    ws_need = max([B.w4a16_workspace_bytes(M, N, K, 128, s) for M, s in zip(SWEEP_M, splits)] + [16384])
     extra_cases = []
     if args.configs:
         for c in wl.CASES:
@@ -229,33 +244,45 @@ def run_ours(args):
         for A, C, s in zip(acts, outs, splits):
             B.w4a16_gemm(A, layer.take(), C, split_k=s)
 
-    launches_per_step = sum(1 + (1 if s > 1 else 0) for s in splits)
+    launches_per_step = len(SWEEP_M)   # one kernel per GEMM: the Split-K reduce is inside it
     step_bytes = sum(wl.algorithmic_bytes(M, K, N) for M in SWEEP_M)
 
-    # ---- main timed region: W warm-up steps, exactly K steps, device events, max over ranks
+    # ---- main timed region: W warm-up steps, exactly K steps, device events, max over ranks.
+    # The steps are captured into CUDA graphs (one rotation through the weight copies each) and
+    # replayed, so the timed region holds exactly steps x 5 kernel launches and no host work.
     for _ in range(args.warmup):
         step()
+    torch.cuda.synchronize()
+    chunk = max(1, min(args.steps, layer.copies))
+    g_main = _capture(step, chunk, torch)
+    reps, rem = divmod(args.steps, chunk)
+    g_rem = _capture(step, rem, torch) if rem else None
+    g_main.replay()
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
-    sampler.start()
+    if not args.no_clocks:
+        sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(args.steps):
-        step()
+    for _ in range(reps):
+        g_main.replay()
+    if g_rem is not None:
+        g_rem.replay()
     e1.record()
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     elapsed = e0.elapsed_time(e1) * 1e-3
-    # keep the sampler alive for at least ~0.5 s of load so that it sees the kernels running
-    t_end = time.perf_counter() + max(0.0, 0.6 - elapsed)
-    while time.perf_counter() < t_end:
-        step()
-    torch.cuda.synchronize()
+    if not args.no_clocks:
+        # keep the same load running until the sampler has seen ~0.6 s of it
+        t_end = time.perf_counter() + max(0.0, 0.6 - elapsed)
+        while time.perf_counter() < t_end:
+            g_main.replay()
+            torch.cuda.synchronize()
     clocks = sampler.stop()
     if dist:
         t = torch.tensor([elapsed], dtype=torch.float64, device="cuda")
@@ -371,6 +398,7 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "group": 128, "accumulate": "f32", "split_k": splits,
                        "l2": "cold: %d packed weight copies (%d MB) rotated, every call reads HBM"
                              % (layer.copies, layer.copies * (K * N // 2) >> 20),
+                       "launch": "CUDA graphs of %d steps, replayed" % chunk,
                        "multi_gpu": "replicas only"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT,
@@ -401,6 +429,7 @@ def main():
     ap.add_argument("--case-calls", type=int, default=400)
     ap.add_argument("--no-cublas", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-clocks", action="store_true", help="do not sample nvidia-smi clocks")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps

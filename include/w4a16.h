@@ -82,7 +82,7 @@ size_t w4a16_packed_z_bytes(int N, int K, int group);
  * w4a16_set_workspace: registers the buffer for the CURRENT device (one per device, per
  * process; replaces the previous one; dev_ptr == NULL, bytes == 0 unregisters).  The
  * buffer must be 256-byte aligned, stays owned by the caller and must outlive every gemm
- * call enqueued while it is registered.  The call zeroes the buffer's first 4 KiB on the
+ * call enqueued while it is registered.  The call zeroes the buffer's first 16 KiB on the
  * default stream and waits for that.  gemm calls that need the workspace and overlap on
  * the GPU (different streams) race on it; serialise them or use split_k = 1. */
 size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k);

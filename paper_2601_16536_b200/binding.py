@@ -187,9 +187,9 @@ def w4a16_gemm_host(A_host: torch.Tensor, A_dev: torch.Tensor, pw: PackedWeights
 def ensure_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     """Allocate (with torch) and register a workspace of at least ``nbytes``; returns the tensor,
     which the caller must keep alive while it is registered."""
-    ws = torch.empty(max(int(nbytes), 4096) + 256, dtype=torch.uint8, device=device)
+    ws = torch.empty(max(int(nbytes), 16384) + 256, dtype=torch.uint8, device=device)
     off = (-ws.data_ptr()) % 256
-    view = ws[off:off + max(int(nbytes), 4096)]
+    view = ws[off:off + max(int(nbytes), 16384)]
     w4a16_set_workspace(view)
     view._keepalive = ws  # type: ignore[attr-defined]
     return view

@@ -14,7 +14,8 @@ using namespace w4a16;
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr size_t kWsHeaderBytes = 4096;  // zeroed control words ahead of the FP32 partials
+constexpr size_t kWsHeaderBytes = 16384;  // zeroed ticket counters ahead of the FP32 partials
+constexpr long kMaxTickets = kWsHeaderBytes / sizeof(int);
 
 struct DeviceState {
     bool probed = false;
@@ -68,58 +69,46 @@ int sm_count_or_default() {
 // ---- decode-path launch geometry ------------------------------------------------
 int decode_mb(int M) { return M <= 8 ? 1 : 2; }
 
+// The decode kernel is persistent: `ctas` CTAs per batch chunk (two per SM: 9 warps and about
+// 100 KiB of shared memory each), `nchunks` chunks of work units dealt to them.
 struct DecodeGeom {
-    int mb, stages, sz_bytes, smem_bytes, ctas_per_sm;
+    int mb, mchunks, stages, smem_bytes, ctas, nchunks;
 };
 
-DecodeGeom decode_geom(int M, int G, int split_k) {
+DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms) {
     DecodeGeom g;
     g.mb = decode_mb(M);
-    int max_ng = (G + split_k - 1) / split_k;
-    g.sz_bytes = ((max_ng * (kSBlockHalves * 2 + kZBlockWords * 4)) + 127) / 128 * 128;
-    int stage = decode_stage_bytes(8 * g.mb);
-    int n_iter = (max_ng + kDecWarps - 1) / kDecWarps;
-    // two CTAs per SM when the ring fits twice in 227 KiB, else one
-    int budget2 = (227 * 1024) / 2 - 1024 - 128 - g.sz_bytes;
-    int budget1 = 227 * 1024 - 1024 - 128 - g.sz_bytes;
-    int st = budget2 / stage;
-    g.ctas_per_sm = 2;
-    if (st < 3) {
-        st = budget1 / stage;
-        g.ctas_per_sm = 1;
-    }
-    if (st > 6) st = 6;
-    if (st > n_iter) st = n_iter;
-    if (st < 1) st = 1;
+    g.mchunks = (M + 8 * g.mb - 1) / (8 * g.mb);
+    const int T = N / kTileN;
+    const long units = (long)T * G;
+    const int budget = (227 * 1024) / 2 - 1024;   // per CTA, two CTAs per SM
+    int st = (budget - 128 - decode_red_bytes(g.mb)) / decode_stage_bytes(g.mb);
+    if (st > kDecMaxStages) st = kDecMaxStages;
+    if (st < 2) st = 2;
     g.stages = st;
-    g.smem_bytes = 128 + g.sz_bytes + st * stage;
+    g.smem_bytes = decode_smem_bytes(g.mb, st);
+    long slots = 2L * sms;
+    if (split_k == 0) {
+        // balanced chunks, one per CTA; no more CTAs than stages' worth of units
+        long want = (units + kDecUnitsPerStage - 1) / kDecUnitsPerStage;
+        g.ctas = (int)(want < slots ? want : slots);
+        if (g.ctas < 1) g.ctas = 1;
+        g.nchunks = g.ctas;
+    } else {
+        g.nchunks = T * split_k;
+        g.ctas = (int)((long)g.nchunks < slots ? (long)g.nchunks : slots);
+    }
     return g;
 }
 
+// Nominal split factor of the balanced schedule: how many CTAs share one column tile's K range.
 int choose_split_decode(int M, int N, int G, int sms) {
-    // Model: CTAs = tiles * m_chunks * S run in waves of (sms * resident CTAs); a CTA's time
-    // is its groups plus a fixed start-up/reduce cost (in units of one group's time).
-    int mb = decode_mb(M);
-    long tiles = (long)(N / kTileN) * ((M + 8 * mb - 1) / (8 * mb));
-    int best = 1;
-    double best_cost = 1e30;
-    for (int s = 1; s <= 16; s *= 2) {
-        if (s > G) break;
-        if (s > 1 && G / s < 2) break;
-        DecodeGeom g = decode_geom(M, G, s);
-        long slots = (long)sms * g.ctas_per_sm;
-        long ctas = tiles * s;
-        long waves = (ctas + slots - 1) / slots;
-        double per_cta = (double)((G + s - 1) / s) + 6.0;
-        // fewer resident CTAs than slots still share the same HBM: scale by occupancy of the last wave
-        double cost = (double)waves * per_cta + (s > 1 ? 2.0 + 0.5 * s : 0.0);
-        if (ctas < slots) cost = per_cta * 1.0 + (s > 1 ? 2.0 + 0.5 * s : 0.0) + (double)(slots - ctas) / slots * 8.0;
-        if (cost < best_cost - 1e-9) {
-            best_cost = cost;
-            best = s;
-        }
-    }
-    return best;
+    DecodeGeom g = decode_geom(M, N, G, 0, sms);
+    const int T = N / kTileN;
+    int s = (g.ctas + T - 1) / T;
+    if (s < 1) s = 1;
+    if (s > G) s = G;
+    return s;
 }
 
 int resolve_path(int M, int path) {
@@ -127,9 +116,15 @@ int resolve_path(int M, int path) {
     return path;
 }
 
-size_t partial_bytes(int M, int N, int split_k) {
-    size_t b = (size_t)split_k * (size_t)M * (size_t)N * sizeof(float);
-    return (b + 255) / 256 * 256;
+size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+
+// FP32 partials of the two-kernel reduce used by the plain path: [split_k][M][N].
+size_t simple_partial_bytes(int M, int N, int split_k) {
+    return round256((size_t)split_k * (size_t)M * (size_t)N * sizeof(float));
+}
+// Partial-tile slots of the decode kernel: [m chunk][2 * nchunks][8 mb][64] FP32.
+size_t decode_partial_bytes(const DecodeGeom& g) {
+    return round256((size_t)g.mchunks * 2 * (size_t)g.nchunks * (8 * g.mb) * kTileN * sizeof(float));
 }
 
 }  // namespace
@@ -179,10 +174,17 @@ int w4a16_choose_split_k(int M, int N, int K, int group) {
 }
 
 size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k) {
-    if (check_weight_shape(N, K, group) != W4A16_OK || M < 1 || split_k < 0) return 0;
-    if (split_k == 0) split_k = w4a16_choose_split_k(M, N, K, group);
-    if (split_k <= 1) return 0;
-    return kWsHeaderBytes + partial_bytes(M, N, split_k);
+    if (check_weight_shape(N, K, group) != W4A16_OK || M < 1 || split_k < 0 || split_k > K / group) return 0;
+    // enough for whichever path w4a16_gemm / w4a16_gemm_ex may take with this split_k
+    size_t need = 0;
+    if (split_k != 1) {
+        DecodeGeom g = decode_geom(M, N, K / group, split_k, sm_count_or_default());
+        need = decode_partial_bytes(g);
+        int s = split_k == 0 ? choose_split_decode(M, N, K / group, sm_count_or_default()) : split_k;
+        size_t simple = simple_partial_bytes(M, N, s);
+        if (simple > need) need = simple;
+    }
+    return need == 0 ? 0 : kWsHeaderBytes + need;
 }
 
 int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
@@ -257,60 +259,60 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
 
     path = resolve_path(M, path);
     if (path == W4A16_PATH_TILE) return W4A16_ERR_PATH;
-    if (split_k == 0) split_k = w4a16_choose_split_k_ex(M, N, K, group, path);
     if (split_k > 65535) return W4A16_ERR_SPLITK;
-
-    float* partials = nullptr;
-    if (split_k > 1) {
-        size_t need = kWsHeaderBytes + partial_bytes(M, N, split_k);
-        if (d->ws == nullptr || d->ws_bytes < need) return W4A16_ERR_WORKSPACE;
-        partials = reinterpret_cast<float*>(static_cast<unsigned char*>(d->ws) + kWsHeaderBytes);
-    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __half* Ah = reinterpret_cast<const __half*>(A);
     __half* Ch = reinterpret_cast<__half*>(C);
+    unsigned char* ws_body = d->ws ? static_cast<unsigned char*>(d->ws) + kWsHeaderBytes : nullptr;
+    const size_t ws_body_bytes = d->ws_bytes > kWsHeaderBytes ? d->ws_bytes - kWsHeaderBytes : 0;
 
     if (path == W4A16_PATH_SIMPLE) {
+        if (split_k == 0) split_k = choose_split_decode(M, N, G, d->sm_count);
+        if (split_k > 1 && ws_body_bytes < simple_partial_bytes(M, N, split_k)) return W4A16_ERR_WORKSPACE;
         int mchunks = (M + kSimpleMB - 1) / kSimpleMB;
         if (mchunks > 65535) return W4A16_ERR_PATH;
+        float* partials = reinterpret_cast<float*>(ws_body);
         dim3 grid(N / kTileN, mchunks, split_k);
         gemm_simple_kernel<<<grid, 64, 0, st>>>(Ah, static_cast<const uint32_t*>(Wq), static_cast<const __half*>(S),
                                                 static_cast<const uint32_t*>(Z), Ch, partials, M, N, K, G, split_k);
-    } else {  // W4A16_PATH_DECODE
-        DecodeGeom g = decode_geom(M, G, split_k);
-        int mchunks = (M + 8 * g.mb - 1) / (8 * g.mb);
-        if (mchunks > 65535) return W4A16_ERR_PATH;
-        if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
-        DecodeParams p;
-        p.A = Ah;
-        p.Wq = static_cast<const uint32_t*>(Wq);
-        p.S = static_cast<const __half*>(S);
-        p.Z = static_cast<const uint32_t*>(Z);
-        p.C = Ch;
-        p.ws = partials;
-        p.M = M; p.N = N; p.K = K; p.G = G;
-        p.split_k = split_k;
-        p.stages = g.stages;
-        p.sz_bytes = g.sz_bytes;
-        auto kern = (g.mb == 1) ? gemm_decode_kernel<1> : gemm_decode_kernel<2>;
-        if (!d->decode_attr_set[g.mb]) {
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return W4A16_ERR_CUDA;
-            }
-            d->decode_attr_set[g.mb] = true;
-        }
-        dim3 grid(N / kTileN, split_k, mchunks);
-        kern<<<grid, kDecThreads, g.smem_bytes, st>>>(p);
-    }
-    if (cudaGetLastError() != cudaSuccess) return W4A16_ERR_CUDA;
-    if (split_k > 1) {
-        size_t MN = (size_t)M * N;
-        splitk_reduce_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, st>>>(partials, Ch, MN, split_k);
         if (cudaGetLastError() != cudaSuccess) return W4A16_ERR_CUDA;
+        if (split_k > 1) {
+            size_t MN = (size_t)M * N;
+            splitk_reduce_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, st>>>(partials, Ch, MN, split_k);
+            if (cudaGetLastError() != cudaSuccess) return W4A16_ERR_CUDA;
+        }
+        return W4A16_OK;
     }
-    return W4A16_OK;
+
+    // W4A16_PATH_DECODE
+    DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count);
+    if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
+    if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
+    if (split_k != 1 && ws_body_bytes < decode_partial_bytes(g)) return W4A16_ERR_WORKSPACE;
+    DecodeParams p;
+    p.A = Ah;
+    p.Wq = static_cast<const uint32_t*>(Wq);
+    p.S = static_cast<const __half*>(S);
+    p.Z = static_cast<const uint32_t*>(Z);
+    p.C = Ch;
+    p.ws = reinterpret_cast<float*>(ws_body);
+    p.tickets = static_cast<int*>(d->ws);
+    p.M = M; p.N = N; p.K = K; p.G = G; p.T = N / kTileN;
+    p.split_k = split_k;
+    p.nchunks = g.nchunks;
+    p.stages = g.stages;
+    auto kern = (g.mb == 1) ? gemm_decode_kernel<1> : gemm_decode_kernel<2>;
+    if (!d->decode_attr_set[g.mb]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return W4A16_ERR_CUDA;
+        }
+        d->decode_attr_set[g.mb] = true;
+    }
+    dim3 grid(g.ctas, g.mchunks, 1);
+    kern<<<grid, kDecThreads, g.smem_bytes, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
 int w4a16_gemm(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,

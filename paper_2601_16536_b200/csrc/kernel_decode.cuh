@@ -1,15 +1,27 @@
-// Small-M ("decode") W4A16 GEMM: bandwidth-bound skinny GEMM.
+// Small-M ("decode") W4A16 GEMM: a persistent, bandwidth-bound skinny GEMM.
 //
-// One CTA owns a 64-column tile of C and one Split-K slice of whole groups.  A producer
-// warp streams the slice's packed blocks (16 KiB = 4 groups per stage, one TMA bulk copy)
-// and the matching activation rows into a multi-stage shared-memory ring guarded by
-// mbarriers.  Four consumer warps each take one group per stage: a 128-bit shared load
-// gives a lane the A-fragment nibbles of a 16-row sub-tile, a logic op and two FP16 ops
-// per register turn them into w16 = fp16_rn((q - z) s), and an m16n8k16 tensor-core MMA
-// with the WEIGHTS as the 16-row operand (MMA rows = n, MMA columns = batch rows)
-// accumulates in FP32.  The four warps' partial sums (disjoint k) are added in warp order
-// through shared memory; the result goes to C (split_k == 1) or to the FP32 Split-K
-// workspace.
+// Work is counted in units: one unit = one packed block = 64 columns x one group (128 k),
+// numbered u = tile * G + group, which is also the block's position in the packed buffers.
+// The unit range [0, T*G) is cut into chunks; a CTA streams its chunk(s) front to back:
+//   - balanced mode (split_k == 0): as many chunks as CTAs, equal to within one unit, so a
+//     chunk may start and end in the middle of a column tile's K range;
+//   - classic Split-K (split_k = S): every tile's K range is cut into S slices of whole
+//     groups (Algorithm 1, Phase 2), T*S chunks dealt round-robin to the CTAs.
+// A producer warp brings 4 units per stage (16 KiB of nibbles + their scales and zeros,
+// three TMA bulk copies) plus the matching activation rows into a shared-memory ring
+// guarded by mbarriers; stages never straddle a tile.  Eight consumer warps work on a
+// stage, two per unit, each on two of the block's four 16-row sub-tiles: a 128-bit shared
+// load gives a lane the A-fragment nibbles, a logic op and two FP16 ops per register turn
+// them into w16 = fp16_rn((q - z) s), and an m16n8k16 tensor-core MMA with the WEIGHTS as
+// the 16-row operand (MMA rows = n, MMA columns = batch rows) accumulates in FP32.
+//
+// When a CTA leaves a tile it adds its warps' sums in a fixed order through shared
+// memory.  If it covered the tile's whole K range it writes FP16 C.  Otherwise it stores
+// the FP32 partial tile in its workspace slot, fences and draws a ticket from the tile's
+// counter; the CTA that draws the last ticket adds the partial tiles in ascending K order,
+// casts to FP16 and writes C (Algorithm 1, Phase 3, inside the same launch).  No CTA
+// waits for another one, and the order of the sum does not depend on which CTA comes
+// last, so results are bit-identical from run to run.
 #pragma once
 
 #include "common.cuh"
@@ -17,11 +29,18 @@
 
 namespace w4a16 {
 
-constexpr int kDecWarps = 4;                       // consumer warps = groups per stage
-constexpr int kDecThreads = (kDecWarps + 1) * 32;  // + producer warp
-constexpr int kDecStageW = kDecWarps * kBlockBytes;             // 16 KiB of packed weights
-constexpr int kDecARowBytes = kDecWarps * kGroup * 2 + 16;      // 1024 B of k + 16 B pad
+constexpr int kDecUnitsPerStage = 4;
+constexpr int kDecWarps = 8;                       // consumer warps (2 per unit of a stage)
+constexpr int kDecConsumers = kDecWarps * 32;
+constexpr int kDecThreads = kDecConsumers + 32;    // + producer warp
+constexpr int kDecMaxStages = 6;
+constexpr int kDecStageW = kDecUnitsPerStage * kBlockBytes;                 // 16384: nibbles
+constexpr int kDecStageS = kDecStageW;                                      // scales at 16384
+constexpr int kDecStageZ = kDecStageS + kDecUnitsPerStage * kSBlockHalves * 2;  // zeros at 16896
+constexpr int kDecStageA = 17152;                                           // activation rows
+constexpr int kDecARowBytes = kDecUnitsPerStage * kGroup * 2 + 16;          // 1024 B of k + 16 B pad
 constexpr int kDecRedStride = 68;                  // floats per batch row in the reduce buffer
+constexpr int kDecUnitBytes = kBlockBytes + kSBlockHalves * 2 + kZBlockWords * 4;  // 4256
 
 struct DecodeParams {
     const __half* A;
@@ -29,14 +48,21 @@ struct DecodeParams {
     const __half* S;
     const uint32_t* Z;
     __half* C;
-    float* ws;       // FP32 partials [split_k][M][N] when split_k > 1
-    int M, N, K, G;
-    int split_k;
+    float* ws;          // partial tiles: [m chunk][2 * nchunks slots][8 MB rows][64] FP32
+    int* tickets;       // zeroed counters: [m chunk][T]
+    int M, N, K, G, T;  // T = N / 64 column tiles
+    int split_k;        // 0: balanced chunks; S >= 1: classic Split-K
+    int nchunks;        // balanced: gridDim.x; classic: T * split_k
     int stages;
-    int sz_bytes;    // shared bytes reserved for the slice's scales + zeros (multiple of 128)
 };
 
-__host__ __device__ inline int decode_stage_bytes(int rows) { return kDecStageW + rows * kDecARowBytes; }
+__host__ __device__ inline int decode_stage_bytes(int mb) { return kDecStageA + 8 * mb * kDecARowBytes; }
+__host__ __device__ inline int decode_red_bytes(int mb) {
+    return kDecUnitsPerStage * 8 * mb * kDecRedStride * 4;
+}
+__host__ __device__ inline int decode_smem_bytes(int mb, int stages) {
+    return 128 + decode_red_bytes(mb) + stages * decode_stage_bytes(mb);
+}
 
 __device__ __forceinline__ void mma_m16n8k16(float (&d)[4], const Frag4& a, uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -47,67 +73,108 @@ __device__ __forceinline__ void mma_m16n8k16(float (&d)[4], const Frag4& a, uint
           "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void consumer_bar() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers) : "memory");
+}
+
+// First unit of chunk i (i == nchunks gives the end of the last chunk).
+__device__ __forceinline__ int chunk_begin(const DecodeParams& p, int i) {
+    if (p.split_k == 0) return (int)(((long long)i * ((long long)p.T * p.G)) / p.nchunks);
+    const int t = i / p.split_k, s = i - t * p.split_k;
+    const int base = p.G / p.split_k, rem = p.G % p.split_k;
+    return t * p.G + s * base + min(s, rem);
+}
+// The chunk that holds unit u.
+__device__ __forceinline__ int chunk_of(const DecodeParams& p, int u) {
+    if (p.split_k == 0) return (int)((((long long)u + 1) * p.nchunks - 1) / ((long long)p.T * p.G));
+    const int t = u / p.G, g = u - t * p.G;
+    const int base = p.G / p.split_k, rem = p.G % p.split_k;
+    // slices 0..rem-1 hold base+1 groups, the rest base groups
+    const int s = (g < rem * (base + 1)) ? g / (base + 1) : rem + (g - rem * (base + 1)) / max(base, 1);
+    return t * p.split_k + s;
+}
+
 // MB = number of 8-row batch blocks one CTA handles (rows m0 .. m0 + 8 MB - 1).
 template <int MB>
 __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    const int t = blockIdx.x, sp = blockIdx.y;
-    const int m0 = blockIdx.z * (8 * MB);
-    const int rows = min(8 * MB, p.M - m0);  // batch rows this CTA really has
+    constexpr int kRows = 8 * MB;
+    const int mz = blockIdx.y;
+    const int m0 = mz * kRows;
+    const int rows = min(kRows, p.M - m0);  // batch rows this CTA really has
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = p.stages;
+    const int stage_bytes = decode_stage_bytes(MB);
 
-    int g0, ng;
-    slice_of(p.G, p.split_k, sp, g0, ng);
-    const int n_iter = (ng + kDecWarps - 1) / kDecWarps;
-
-    // shared layout: [barriers 128 B][S slice | Z slice][stage 0][stage 1]...
+    // shared layout: [barriers + flag, 128 B][reduce buffer][stage 0][stage 1]...
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);
-    uint64_t* empty = full + 6;
-    uint64_t* szbar = full + 12;
-    unsigned char* sz = smem + 128;
-    const __half* s_s = reinterpret_cast<const __half*>(sz);
-    const uint32_t* z_s = reinterpret_cast<const uint32_t*>(sz + ng * (kSBlockHalves * 2));
-    unsigned char* stage0 = sz + p.sz_bytes;
-    const int stage_bytes = decode_stage_bytes(8 * MB);
+    uint64_t* empty = full + kDecMaxStages;
+    int* last_flag = reinterpret_cast<int*>(smem + 120);
+    float* red = reinterpret_cast<float*>(smem + 128);
+    unsigned char* stage0 = smem + 128 + decode_red_bytes(MB);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
             mbar_init(&full[i], 1);
             mbar_init(&empty[i], kDecWarps);
         }
-        mbar_init(szbar, 1);
         fence_mbar_init();
     }
+    // activation rows this CTA does not have stay zero for the whole kernel
+    if (rows < kRows) {
+        for (int s = 0; s < stages; ++s) {
+            uint32_t* z = reinterpret_cast<uint32_t*>(stage0 + (size_t)s * stage_bytes + kDecStageA +
+                                                      rows * kDecARowBytes);
+            for (int i = threadIdx.x; i < (kRows - rows) * kDecARowBytes / 4; i += kDecThreads) z[i] = 0u;
+        }
+    }
     __syncthreads();
-
-    const size_t blk0 = (size_t)t * p.G + g0;  // first packed block of the slice
+    // Let the next kernel in the stream start its own prologue; everything below that reads
+    // or writes memory another kernel may have written comes after griddepcontrol.wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kDecWarps) {
         // ------------------------------------------------ producer warp
-        if (lane == 0) {
-            mbar_expect_tx(szbar, (uint32_t)(ng * (kSBlockHalves * 2 + kZBlockWords * 4)));
-            bulk_g2s(sz, p.S + blk0 * kSBlockHalves, (uint32_t)(ng * kSBlockHalves * 2), szbar);
-            bulk_g2s(sz + ng * (kSBlockHalves * 2), p.Z + blk0 * kZBlockWords, (uint32_t)(ng * kZBlockWords * 4),
-                     szbar);
-        }
-        for (int it = 0; it < n_iter; ++it) {
-            const int s = it % stages;
-            const int gc = min(kDecWarps, ng - it * kDecWarps);
-            bool ok = true;
-            if (it >= stages) ok = mbar_wait(&empty[s], (uint32_t)((it / stages - 1) & 1));
-            if (!ok) break;  // status recorded; consumers will time out too and the CTA ends
-            unsigned char* st = stage0 + (size_t)s * stage_bytes;
-            if (lane == 0) {
-                mbar_expect_tx(&full[s], (uint32_t)(gc * kBlockBytes + rows * gc * (kGroup * 2)));
-                bulk_g2s(st, p.Wq + (blk0 + (size_t)it * kDecWarps) * kBlockWords, (uint32_t)(gc * kBlockBytes),
-                         &full[s]);
-            }
-            __syncwarp();
-            for (int m = lane; m < rows; m += 32) {
-                bulk_g2s(st + kDecStageW + m * kDecARowBytes,
-                         p.A + (size_t)(m0 + m) * p.K + (size_t)(g0 + it * kDecWarps) * kGroup,
-                         (uint32_t)(gc * kGroup * 2), &full[s]);
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        int slot = 0;
+        uint32_t phase = 0;
+        bool first_round = true;
+        for (int ci = blockIdx.x; ci < p.nchunks; ci += gridDim.x) {
+            int u = chunk_begin(p, ci);
+            const int u1 = chunk_begin(p, ci + 1);
+            if (u >= u1) continue;
+            int t = u / p.G;
+            int tile_end = (t + 1) * p.G;
+            while (u < u1) {
+                const int gc = min(kDecUnitsPerStage, min(u1, tile_end) - u);
+                if (!first_round) {
+                    if (!mbar_wait(&empty[slot], phase ^ 1u)) return;  // status recorded
+                }
+                unsigned char* st = stage0 + (size_t)slot * stage_bytes;
+                if (lane == 0) {
+                    mbar_expect_tx(&full[slot], (uint32_t)(gc * kDecUnitBytes + rows * gc * (kGroup * 2)));
+                    bulk_g2s(st, p.Wq + (size_t)u * kBlockWords, (uint32_t)(gc * kBlockBytes), &full[slot]);
+                    bulk_g2s(st + kDecStageS, p.S + (size_t)u * kSBlockHalves, (uint32_t)(gc * kSBlockHalves * 2),
+                             &full[slot]);
+                    bulk_g2s(st + kDecStageZ, p.Z + (size_t)u * kZBlockWords, (uint32_t)(gc * kZBlockWords * 4),
+                             &full[slot]);
+                }
+                __syncwarp();
+                const int g = u - t * p.G;  // the stage's units are groups g .. g + gc - 1 of tile t
+                for (int m = lane; m < rows; m += 32) {
+                    bulk_g2s(st + kDecStageA + m * kDecARowBytes, p.A + (size_t)(m0 + m) * p.K + (size_t)g * kGroup,
+                             (uint32_t)(gc * kGroup * 2), &full[slot]);
+                }
+                u += gc;
+                if (u == tile_end) {
+                    ++t;
+                    tile_end += p.G;
+                }
+                if (++slot == stages) {
+                    slot = 0;
+                    phase ^= 1u;
+                    first_round = false;
+                }
             }
         }
         return;
@@ -115,102 +182,147 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
 
     // ---------------------------------------------------- consumer warps
     const int gq = lane >> 2, tig = lane & 3;
-    float acc[4][MB][4];
+    const int us = warp >> 1;         // which unit of the stage
+    const int r0 = (warp & 1) * 2;    // first of this warp's two 16-row sub-tiles
+    float acc[2][MB][4];
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
+    for (int r = 0; r < 2; ++r)
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[r][mb][i] = 0.f;
 
-    bool alive = mbar_wait(szbar, 0);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float* const ws_mz = p.ws + (size_t)mz * (2 * (size_t)p.nchunks) * (kRows * kTileN);
+    int* const tickets_mz = p.tickets + (size_t)mz * p.T;
 
-    for (int it = 0; it < n_iter && alive; ++it) {
-        const int s = it % stages;
-        alive = mbar_wait(&full[s], (uint32_t)((it / stages) & 1));
-        if (!alive) break;
-        const int gc = min(kDecWarps, ng - it * kDecWarps);
-        if (warp < gc) {
-            const int lg = it * kDecWarps + warp;  // group index inside the slice
-            const unsigned char* st = stage0 + (size_t)s * stage_bytes;
-            const uint4* wsm = reinterpret_cast<const uint4*>(st + warp * kBlockBytes);
-            const unsigned char* asm_ = st + kDecStageW + warp * (kGroup * 2);
+    int slot = 0;
+    uint32_t phase = 0;
+    for (int ci = blockIdx.x; ci < p.nchunks; ci += gridDim.x) {
+        const int u0 = chunk_begin(p, ci);
+        const int u1 = chunk_begin(p, ci + 1);
+        if (u0 >= u1) continue;
+        int u = u0;
+        int t = u / p.G;
+        int tile_end = (t + 1) * p.G;
+        int seg_start = u0;
+        while (u < u1) {
+            const int gc = min(kDecUnitsPerStage, min(u1, tile_end) - u);
+            if (!mbar_wait(&full[slot], phase)) return;  // status recorded; every consumer warp sees it
+            if (us < gc) {
+                const unsigned char* st = stage0 + (size_t)slot * stage_bytes;
+                const uint4* wsm = reinterpret_cast<const uint4*>(st + us * kBlockBytes);
+                const unsigned char* a_s = st + kDecStageA + us * (kGroup * 2);
 
-            // scales / zero points of this lane's 8 rows (16r + gq + 8h)
-            uint4 sraw = *reinterpret_cast<const uint4*>(s_s + lg * kSBlockHalves + gq * 8);
-            const uint32_t zw = z_s[lg * kZBlockWords + gq];
-            const uint32_t sw[4] = {sraw.x, sraw.y, sraw.z, sraw.w};
-
-            __half2 s_lo[4], s_hi[4], zlo[4], zhi[4];
+                // scales / zero points of this lane's rows 16r + gq + 8h, r = r0, r0 + 1
+                const uint2 sraw = *reinterpret_cast<const uint2*>(st + kDecStageS + us * (kSBlockHalves * 2) +
+                                                                   gq * 16 + r0 * 4);
+                const uint32_t zw =
+                    *reinterpret_cast<const uint32_t*>(st + kDecStageZ + us * (kZBlockWords * 4) + gq * 4) >> (8 * r0);
+                const uint32_t sw[2] = {sraw.x, sraw.y};
+                __half2 s_lo[2], s_hi[2], zlo[2], zhi[2];
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                s_lo[r] = __half2half2(__low2half(u32_as_h2(sw[r])));   // row 16r + gq
-                s_hi[r] = __half2half2(__high2half(u32_as_h2(sw[r])));  // row 16r + gq + 8
-                zlo[r] = u32_as_h2(zmagic_lo((zw >> (8 * r)) & 15u));
-                zhi[r] = u32_as_h2(zmagic_hi((zw >> (8 * r + 4)) & 15u));
-            }
-
+                for (int r = 0; r < 2; ++r) {
+                    s_lo[r] = __half2half2(__low2half(u32_as_h2(sw[r])));   // row 16(r0+r) + gq
+                    s_hi[r] = __half2half2(__high2half(u32_as_h2(sw[r])));  // row 16(r0+r) + gq + 8
+                    zlo[r] = u32_as_h2(zmagic_lo((zw >> (8 * r)) & 15u));
+                    zhi[r] = u32_as_h2(zmagic_hi((zw >> (8 * r + 4)) & 15u));
+                }
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                // B fragments: batch row 8 mb + gq, 16 consecutive k per lane
-                uint32_t bw[MB][8];
+                for (int c = 0; c < 2; ++c) {
+                    // B fragments: batch row 8 mb + gq, 16 consecutive k per lane
+                    uint32_t bw[MB][8];
 #pragma unroll
-                for (int mb = 0; mb < MB; ++mb) {
-                    if (mb * 8 + gq < rows) {
+                    for (int mb = 0; mb < MB; ++mb) {
                         const uint4* ap =
-                            reinterpret_cast<const uint4*>(asm_ + (mb * 8 + gq) * kDecARowBytes + c * 128 + tig * 32);
-                        uint4 x = ap[0], y = ap[1];
+                            reinterpret_cast<const uint4*>(a_s + (mb * 8 + gq) * kDecARowBytes + c * 128 + tig * 32);
+                        const uint4 x = ap[0], y = ap[1];
                         bw[mb][0] = x.x; bw[mb][1] = x.y; bw[mb][2] = x.z; bw[mb][3] = x.w;
                         bw[mb][4] = y.x; bw[mb][5] = y.y; bw[mb][6] = y.z; bw[mb][7] = y.w;
-                    } else {
+                    }
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) bw[mb][i] = 0u;
+                    for (int r = 0; r < 2; ++r) {
+                        const uint4 wv = wsm[(c * 4 + r0 + r) * 32 + lane];
+                        const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const Frag4 f = dequant_word(ww[j], zlo[r], zhi[r], s_lo[r], s_hi[r]);
+#pragma unroll
+                            for (int mb = 0; mb < MB; ++mb)
+                                mma_m16n8k16(acc[r][mb], f, bw[mb][2 * j], bw[mb][2 * j + 1]);
+                        }
                     }
                 }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[slot]);
+            if (++slot == stages) {
+                slot = 0;
+                phase ^= 1u;
+            }
+            u += gc;
+            if (u != tile_end && u != u1) continue;
+
+            // ------------------------------------------------ leave tile t: units [seg_start, u)
+            consumer_bar();
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const uint4 wv = wsm[(c * 4 + r) * 32 + lane];
-                    const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+            for (int r = 0; r < 2; ++r)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const Frag4 f = dequant_word(ww[j], zlo[r], zhi[r], s_lo[r], s_hi[r]);
+                for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
-                        for (int mb = 0; mb < MB; ++mb) mma_m16n8k16(acc[r][mb], f, bw[mb][2 * j], bw[mb][2 * j + 1]);
+                    for (int i = 0; i < 4; ++i) {
+                        const int n = (r0 + r) * 16 + gq + (i >= 2 ? 8 : 0);
+                        const int m = mb * 8 + 2 * tig + (i & 1);
+                        red[(us * kRows + m) * kDecRedStride + n] = acc[r][mb][i];
+                        acc[r][mb][i] = 0.f;
+                    }
+            consumer_bar();
+            const int tile_u0 = t * p.G;
+            const bool whole = (seg_start == tile_u0) && (u == tile_end);
+            // first segment of a chunk -> slot 2 ci, a chunk's continuation into a later tile -> 2 ci + 1
+            float* my_slot = ws_mz + (size_t)(2 * ci + (seg_start == u0 ? 0 : 1)) * (kRows * kTileN);
+            for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
+                const int n = idx & (kTileN - 1), m = idx >> 6;
+                float v = red[m * kDecRedStride + n];
+#pragma unroll
+                for (int w = 1; w < kDecUnitsPerStage; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
+                if (whole)
+                    p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
+                else
+                    my_slot[idx] = v;
+            }
+            if (!whole) {
+                __threadfence();  // this thread's partial stores are visible device-wide before the ticket
+                consumer_bar();
+                const int c_first = chunk_of(p, tile_u0);
+                const int c_last = chunk_of(p, tile_end - 1);
+                if (threadIdx.x == 0) {
+                    const int old = atomicAdd(&tickets_mz[t], 1);
+                    const int last = (old == c_last - c_first);
+                    if (last) tickets_mz[t] = 0;  // all contributors have arrived: zero for the next call
+                    *last_flag = last;
+                }
+                consumer_bar();
+                if (*last_flag) {
+                    __threadfence();
+                    // contributors in ascending K: chunk c_first (its first segment if it starts at the
+                    // tile's first unit, else its continuation), then the first segments of the others
+                    const int first_slot = 2 * c_first + (chunk_begin(p, c_first) == tile_u0 ? 0 : 1);
+                    for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
+                        const int n = idx & (kTileN - 1), m = idx >> 6;
+                        float v = __ldcg(ws_mz + (size_t)first_slot * (kRows * kTileN) + idx);
+                        for (int c = c_first + 1; c <= c_last; ++c)
+                            v += __ldcg(ws_mz + (size_t)(2 * c) * (kRows * kTileN) + idx);
+                        p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
                     }
                 }
+            }
+            seg_start = u;
+            if (u == tile_end) {
+                ++t;
+                tile_end += p.G;
             }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);
-    }
-
-    // ---------------------------------------------------- cross-warp sum (fixed order)
-    // All copies this CTA issued have been consumed, so stage memory is free to reuse.
-    float* red = reinterpret_cast<float*>(stage0);
-    constexpr int kRows = 8 * MB;
-    asm volatile("bar.sync 1, %0;" ::"n"(kDecWarps * 32) : "memory");
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                int n = r * 16 + gq + (i >= 2 ? 8 : 0);
-                int m = mb * 8 + 2 * tig + (i & 1);
-                red[(warp * kRows + m) * kDecRedStride + n] = acc[r][mb][i];
-            }
-    asm volatile("bar.sync 1, %0;" ::"n"(kDecWarps * 32) : "memory");
-    if (!alive) return;
-    for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecWarps * 32) {
-        int n = idx & (kTileN - 1), m = idx >> 6;
-        float v = red[m * kDecRedStride + n];
-#pragma unroll
-        for (int w = 1; w < kDecWarps; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
-        size_t off = (size_t)(m0 + m) * p.N + (size_t)t * kTileN + n;
-        if (p.split_k == 1)
-            p.C[off] = __float2half_rn(v);
-        else
-            p.ws[(size_t)sp * p.M * p.N + off] = v;
     }
 }
 

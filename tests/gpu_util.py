@@ -41,5 +41,6 @@ def assert_close(C_gpu: np.ndarray, C_ref: np.ndarray, what=""):
 
 
 def ensure_ws(M, N, K, split_k, group=128):
-    need = max(B.w4a16_workspace_bytes(M, N, K, group, split_k), 4096)
+    splits = split_k if isinstance(split_k, (tuple, list)) else (split_k,)
+    need = max([B.w4a16_workspace_bytes(M, N, K, group, s) for s in splits] + [16384])
     return B.ensure_workspace(need)

@@ -52,8 +52,9 @@ def test_choose_split_k_is_always_acceptable(lib):
             for path in (1, 2, 3):
                 s = lib.w4a16_choose_split_k_ex(M, N, K, 128, path)
                 assert 1 <= s <= K // 128
-            ws = lib.w4a16_workspace_bytes(M, N, K, 128, 0)
-            assert ws == lib.w4a16_workspace_bytes(M, N, K, 128, lib.w4a16_choose_split_k(M, N, K, 128))
+            # automatic scheduling shares column tiles between CTAs, so it needs partial-tile slots
+            assert lib.w4a16_workspace_bytes(M, N, K, 128, 0) >= 16384
+            assert lib.w4a16_workspace_bytes(M, N, K, 128, 1) == 0
     assert lib.w4a16_workspace_bytes(4, 4096, 4096, 128, 1) == 0
     assert lib.w4a16_workspace_bytes(4, 4096, 4096, 128, 4) >= 4 * 4 * 4096 * 4
 

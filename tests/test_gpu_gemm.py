@@ -20,7 +20,7 @@ PATHS = {"simple": B.PATH_SIMPLE, "decode": B.PATH_DECODE}
 
 def _run(d, M, N, K, split_k, path):
     pw = pack_problem(d, N, K)
-    ws = ensure_ws(M, N, K, split_k if split_k else B.w4a16_choose_split_k(M, N, K, 128, path))
+    ws = ensure_ws(M, N, K, split_k)
     C = B.w4a16_gemm(to_dev(d["A"]), pw, split_k=split_k, path=path)
     torch.cuda.synchronize()
     assert B.w4a16_device_status() == 0
@@ -36,7 +36,7 @@ SMALL = [(1, 128, 64), (1, 640, 192), (3, 896, 128), (8, 1152, 256), (9, 640, 12
 
 @pytest.mark.parametrize("path", list(PATHS))
 @pytest.mark.parametrize("M,K,N", SMALL)
-@pytest.mark.parametrize("split_k", [1, 2, 3])
+@pytest.mark.parametrize("split_k", [0, 1, 2, 3])
 def test_small_shapes_match_oracle(path, M, K, N, split_k):
     if split_k > K // 128:
         pytest.skip("more splits than groups")
@@ -63,7 +63,7 @@ def test_exact_inputs_are_bit_equal_for_every_split(path):
     M, K, N = 7, 2304, 192    # 18 groups
     d = wl.make_exact_problem(M, K, N, seed=90)
     want = oracle.gemm_int(d["A_int"], d["Wq"], d["E"], d["Z"], M, N, K, 128)
-    for split_k in (1, 2, 4, 5, 8, 16, 18):
+    for split_k in (0, 1, 2, 4, 5, 8, 16, 18):
         C = _run(d, M, N, K, split_k, PATHS[path])
         assert np.array_equal(c_bits(C), want), "split_k=%d" % split_k
 
@@ -88,8 +88,8 @@ def test_results_are_bit_identical_run_to_run():
     d = wl.make_problem(M, K, N, seed=92)
     pw = pack_problem(d, N, K)
     A = to_dev(d["A"])
-    ws = ensure_ws(M, N, K, 16)
-    for split_k in (1, 4, 16):
+    ws = ensure_ws(M, N, K, (0, 16))
+    for split_k in (0, 1, 4, 16):
         first = c_bits(B.w4a16_gemm(A, pw, split_k=split_k, path=B.PATH_DECODE))
         for _ in range(5):
             again = c_bits(B.w4a16_gemm(A, pw, split_k=split_k, path=B.PATH_DECODE))
@@ -114,8 +114,8 @@ def test_workspace_errors():
     with pytest.raises(B.W4A16Error) as e:
         B.w4a16_gemm(A, pw, split_k=4, path=B.PATH_DECODE)
     assert e.value.code == -5
-    small = torch.empty(8192, dtype=torch.uint8, device="cuda")
-    B.w4a16_set_workspace(small[(-small.data_ptr()) % 256:][:4096 + 256])
+    small = torch.empty(32768, dtype=torch.uint8, device="cuda")
+    B.w4a16_set_workspace(small[(-small.data_ptr()) % 256:][:16384 + 256])
     with pytest.raises(B.W4A16Error) as e:
         B.w4a16_gemm(A, pw, split_k=4, path=B.PATH_DECODE)
     assert e.value.code == -5
