@@ -229,7 +229,7 @@ def run_ours(args):
     acts_np = [wl.draw_activations(M, K, 2000 + i) for i, M in enumerate(SWEEP_M)]
     acts = [_to_dev(a, torch) for a in acts_np]
     outs = [torch.empty((M, N), dtype=torch.float16, device="cuda") for M in SWEEP_M]
-    splits = [args.split_k if args.split_k else B.w4a16_choose_split_k(M, N, K) for M in SWEEP_M]
+    splits = [args.split_k for M in SWEEP_M]   # 0 = the library's own schedule
     ws_need = max([B.w4a16_workspace_bytes(M, N, K, 128, s) for M, s in zip(SWEEP_M, splits)] + [16384])
     extra_cases = []
     if args.configs:
@@ -331,7 +331,7 @@ def run_ours(args):
             cur = Layer(c.K, c.N, c.seed, torch, B, wl)
         A = _to_dev(wl.draw_activations(c.M, c.K, c.seed, c.a_sigma, c.outliers), torch)
         C = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
-        s = B.w4a16_choose_split_k(c.M, c.N, c.K)
+        s = 0
         sec = _time_calls(lambda: B.w4a16_gemm(A, cur.take(), C, split_k=s), 10,
                           max(20, args.case_calls // 4), torch)
         byts = wl.algorithmic_bytes(c.M, c.K, c.N)
@@ -417,6 +417,37 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_one(args):
+    """One shape alone: `--one M,K,N` packs rotating weight copies, makes --calls plain stream
+    launches (no CUDA graph) and prints the mean device time per call.  The small, launch-by-launch
+    command used for profiler captures."""
+    import torch
+    from paper_2601_16536_b200 import binding as B
+    from paper_2601_16536_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    M, K, N = args.one
+    layer = Layer(K, N, 1, torch, B, wl, min_bytes=args.rotation_mb << 20)
+    A = _to_dev(wl.draw_activations(M, K, 1), torch)
+    C = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    ws = B.ensure_workspace(max(B.w4a16_workspace_bytes(M, N, K, 128, args.split_k), 16384))
+    for _ in range(3):
+        B.w4a16_gemm(A, layer.take(), C, split_k=args.split_k, path=args.path)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.calls):
+        B.w4a16_gemm(A, layer.take(), C, split_k=args.split_k, path=args.path)
+    e1.record()
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    us = e0.elapsed_time(e1) * 1e3 / args.calls
+    byts = wl.algorithmic_bytes(M, K, N)
+    print(json.dumps({"one": [M, K, N], "path": args.path, "split_k": args.split_k, "calls": args.calls,
+                      "us_per_call_stream": us, "eff_GBps": byts / us / 1e3,
+                      "tflops": 2.0 * M * N * K / us / 1e6, "copies": layer.copies}))
+    del ws
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -430,7 +461,15 @@ def main():
     ap.add_argument("--no-cublas", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-clocks", action="store_true", help="do not sample nvidia-smi clocks")
+    ap.add_argument("--one", type=lambda s: [int(x) for x in s.split(",")], default=None,
+                    help="M,K,N: time this one shape with plain stream launches and exit")
+    ap.add_argument("--calls", type=int, default=20, help="launches of --one")
+    ap.add_argument("--path", type=int, default=0, help="kernel path of --one (0 auto, 1 simple, 2 decode, 3 tile)")
+    ap.add_argument("--rotation-mb", type=int, default=512, help="bytes of rotating weight copies of --one")
     args = ap.parse_args()
+    if args.one:
+        run_one(args)
+        return
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
