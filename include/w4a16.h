@@ -135,6 +135,37 @@ int w4a16_gemm_host(const uint16_t *A_host, uint16_t *A_dev, const void *Wq, con
                     const void *Z, uint16_t *C_dev, uint16_t *C_host, int M, int N, int K,
                     int group, int split_k, w4a16_stream_t stream);
 
+/* No counterpart in the paper: an extra entry point for callers that must not allocate.
+ *
+ * Some hosts of this library cannot hand it a workspace: an inference runtime that sizes all
+ * of its device memory at start-up and forbids cudaMalloc afterwards (an allocation stalls the
+ * whole device), a plug-in that runs inside someone else's memory pool, a control loop with a
+ * latency bound, or code on a path where the allocator may not be entered at all.  For them
+ * this call computes the same product as w4a16_gemm on the small-M kernel (the one whose
+ * Split-K keeps FP32 partial tiles and ticket counters in scratch memory), but takes that
+ * scratch from an array of W4A16_STATIC_WS_BYTES bytes built into the library's device image
+ * instead of the buffer registered with w4a16_set_workspace.  It calls no cudaMalloc, no
+ * cudaFree and no allocating library routine; A, Wq, S, Z and C are still the caller's.
+ *
+ *   - Cost: every GPU on which the library is loaded holds the W4A16_STATIC_WS_BYTES until the
+ *     process exits, whether or not this call is ever made.
+ *   - Limit: a shape / split_k whose scratch need (16 KiB of counters + the partial tiles, the
+ *     same amount w4a16_workspace_bytes reports for the small-M kernel) exceeds the array is
+ *     rejected with W4A16_ERR_WORKSPACE and nothing is launched.  Every M <= 16 with
+ *     split_k = 0 fits; large explicit split_k on wide N may not.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current) and sets a kernel attribute; make that
+ *     first call outside any stream capture.  Later calls only enqueue work.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.
+ *     Each call first clears the counter block with a cudaMemsetAsync on `stream`, then
+ *     launches the kernel.  Two calls that overlap on the GPU (different streams, or this call
+ *     from two threads) race on the array: keep them ordered.
+ *   - Arguments, preconditions, result and error codes are otherwise those of w4a16_gemm. */
+#define W4A16_STATIC_WS_BYTES (4u * 1024u * 1024u + 16384u)
+int w4a16_gemm_static_ws(const uint16_t *A, const void *Wq, const void *S, const void *Z,
+                         uint16_t *C, int M, int N, int K, int group, int split_k,
+                         w4a16_stream_t stream);
+
 /* Kernels never wait without a limit: a wait that runs out records a code in a status
  * word on the device and the kernel returns.  This call synchronises the current
  * device, copies the word to *status_out (0 = no kernel ever gave up) and clears it.

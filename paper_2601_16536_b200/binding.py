@@ -24,7 +24,7 @@ EXPORTS = (
     "w4a16_strerror", "w4a16_packed_wq_bytes", "w4a16_packed_s_bytes", "w4a16_packed_z_bytes",
     "w4a16_workspace_bytes", "w4a16_set_workspace", "w4a16_choose_split_k",
     "w4a16_choose_split_k_ex", "w4a16_pack", "w4a16_dequant", "w4a16_gemm", "w4a16_gemm_ex",
-    "w4a16_gemm_host", "w4a16_device_status",
+    "w4a16_gemm_host", "w4a16_gemm_static_ws", "w4a16_device_status",
 )
 
 _lib = None
@@ -70,6 +70,8 @@ def load():
     L.w4a16_gemm_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, vp]
     L.w4a16_gemm_host.restype = i
     L.w4a16_gemm_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    L.w4a16_gemm_static_ws.restype = i
+    L.w4a16_gemm_static_ws.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.w4a16_device_status.restype = i
     L.w4a16_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
     _lib = L
@@ -182,6 +184,20 @@ def w4a16_gemm_host(A_host: torch.Tensor, A_dev: torch.Tensor, pw: PackedWeights
     _check(load().w4a16_gemm_host(_ptr(A_host), _ptr(A_dev), _ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z),
                                   _ptr(C_dev), _ptr(C_host), M, pw.N, pw.K, pw.group, split_k,
                                   _stream()), "w4a16_gemm_host")
+
+
+def w4a16_gemm_static_ws(A: torch.Tensor, pw: PackedWeights, C: Optional[torch.Tensor] = None,
+                         split_k: int = 0) -> torch.Tensor:
+    """``w4a16_gemm`` for callers that may not allocate: the Split-K scratch is an array built into
+    the library, nothing is registered and the library allocates nothing.  Pass ``C`` to keep this
+    wrapper from allocating the output as well.  Calls that overlap on the GPU race on the shared
+    array; shapes whose scratch need exceeds it raise ``W4A16Error`` (-5)."""
+    M = A.shape[0]
+    if C is None:
+        C = torch.empty((M, pw.N), dtype=torch.float16, device=A.device)
+    _check(load().w4a16_gemm_static_ws(_ptr(A), _ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(C), M, pw.N,
+                                       pw.K, pw.group, split_k, _stream()), "w4a16_gemm_static_ws")
+    return C
 
 
 def ensure_workspace(nbytes: int, device="cuda") -> torch.Tensor:

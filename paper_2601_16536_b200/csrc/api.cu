@@ -127,6 +127,13 @@ size_t decode_partial_bytes(const DecodeGeom& g) {
     return round256((size_t)g.mchunks * 2 * (size_t)g.nchunks * (8 * g.mb) * kTileN * sizeof(float));
 }
 
+// ---- built-in scratch for w4a16_gemm_static_ws -------------------------------------
+// Lives in the library's device image: every GPU that loads the library holds these bytes until
+// the process exits.  In host code `g_static_ws` is only a handle for cudaGetSymbolAddress; the
+// device address is looked up once per device (below) and that is what the kernel receives.
+static __device__ __align__(256) unsigned char g_static_ws[W4A16_STATIC_WS_BYTES];
+unsigned char* g_static_ws_addr[kMaxDevices] = {};
+
 }  // namespace
 
 // =====================================================================================
@@ -337,6 +344,68 @@ int w4a16_gemm_host(const uint16_t* A_host, uint16_t* A_dev, const void* Wq, con
         return W4A16_ERR_CUDA;
     }
     return W4A16_OK;
+}
+
+int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N,
+                         int K, int group, int split_k, w4a16_stream_t stream) {
+    if (!A || !Wq || !S || !Z || !C) return W4A16_ERR_NULL;
+    int rc = check_weight_shape(N, K, group);
+    if (rc != W4A16_OK) return rc;
+    if (M < 1) return W4A16_ERR_SHAPE;
+    if (!aligned16(A) || !aligned16(Wq) || !aligned16(S) || !aligned16(Z) || !aligned16(C)) return W4A16_ERR_ALIGN;
+    const int G = K / group;
+    if (split_k < 0 || split_k > G) return W4A16_ERR_SPLITK;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != W4A16_OK) return rc;
+    if (!d->is_sm100) return W4A16_ERR_ARCH;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return W4A16_ERR_CUDA;
+
+    const DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count);
+    if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
+    if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
+    // the whole scratch need of this shape must fit the built-in array, or nothing is launched
+    if (kWsHeaderBytes + decode_partial_bytes(g) > (size_t)W4A16_STATIC_WS_BYTES) return W4A16_ERR_WORKSPACE;
+
+    // first call on this device: resolve the array's device address (this device is current)
+    if (g_static_ws_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return W4A16_ERR_CUDA;
+        }
+        g_static_ws_addr[dev] = static_cast<unsigned char*>(p);
+    }
+    unsigned char* ws = g_static_ws_addr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left; the ticket counters must start at zero
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) {
+        cudaGetLastError();
+        return W4A16_ERR_CUDA;
+    }
+    DecodeParams p;
+    p.A = reinterpret_cast<const __half*>(A);
+    p.Wq = static_cast<const uint32_t*>(Wq);
+    p.S = static_cast<const __half*>(S);
+    p.Z = static_cast<const uint32_t*>(Z);
+    p.C = reinterpret_cast<__half*>(C);
+    p.ws = reinterpret_cast<float*>(ws + kWsHeaderBytes);
+    p.tickets = reinterpret_cast<int*>(ws);
+    p.M = M; p.N = N; p.K = K; p.G = G; p.T = N / kTileN;
+    p.split_k = split_k;
+    p.nchunks = g.nchunks;
+    p.stages = g.stages;
+    auto kern = (g.mb == 1) ? gemm_decode_kernel<1> : gemm_decode_kernel<2>;
+    if (!d->decode_attr_set[g.mb]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return W4A16_ERR_CUDA;
+        }
+        d->decode_attr_set[g.mb] = true;
+    }
+    kern<<<dim3(g.ctas, g.mchunks, 1), kDecThreads, g.smem_bytes, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
 int w4a16_device_status(int* status_out) {
