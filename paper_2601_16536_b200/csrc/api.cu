@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "kernels_basic.cuh"
 #include "kernel_decode.cuh"
+#include "kernel_tile.cuh"
 
 using namespace w4a16;
 
@@ -25,6 +26,7 @@ struct DeviceState {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     bool decode_attr_set[3] = {false, false, false};
+    bool tile_attr_set[4] = {false, false, false, false};
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -59,6 +61,8 @@ int check_weight_shape(int N, int K, int group) {
     if (K <= 0 || N <= 0 || K % kGroup != 0 || N % kTileN != 0) return W4A16_ERR_SHAPE;
     return W4A16_OK;
 }
+
+size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 
 int sm_count_or_default() {
     DeviceState* d = nullptr;
@@ -111,12 +115,95 @@ int choose_split_decode(int M, int N, int G, int sms) {
     return s;
 }
 
-int resolve_path(int M, int path) {
-    if (path == W4A16_PATH_AUTO) return W4A16_PATH_DECODE;
-    return path;
+// ---- tile-path launch geometry ----------------------------------------------------
+// MT (batch rows per CTA tile = UMMA N) is the smallest of 32, 64, 128, 256 that covers M, else 256.
+struct TileGeom {
+    int mt, mt_index, m_tiles, n_tiles, split_k, stages, smem_bytes, ctas;
+    long items;
+};
+
+int tile_mt_index(int M) { return M <= 32 ? 0 : M <= 64 ? 1 : M <= 128 ? 2 : 3; }
+
+// Split factor of the tile path when the caller leaves it open (the paper takes S as an input).
+// Cost model: the grid runs ceil(tiles * S / SMs) waves, each as long as one item: ceil(G / S)
+// groups of main loop plus a fixed part (pipeline fill, epilogue, partial-tile exchange) worth
+// about six groups.  Slices keep at least four groups; S <= 16; S = 1 once the tiles fill the SMs.
+int choose_split_tile(int M, int N, int G, int sms) {
+    const int mt = 32 << tile_mt_index(M);
+    const long tiles = (long)((N + kTileCols - 1) / kTileCols) * ((M + mt - 1) / mt);
+    int best = 1;
+    long best_cost = -1;
+    for (int s = 1; s <= 16 && (s == 1 || G / s >= 4); ++s) {
+        const long waves = (tiles * s + sms - 1) / sms;
+        const long cost = waves * ((G + s - 1) / s + (s > 1 ? 6 : 4));
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    return best;
 }
 
-size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
+    TileGeom g;
+    g.mt_index = tile_mt_index(M);
+    g.mt = 32 << g.mt_index;
+    g.m_tiles = (M + g.mt - 1) / g.mt;
+    g.n_tiles = (N + kTileCols - 1) / kTileCols;
+    g.split_k = split_k == 0 ? choose_split_tile(M, N, G, sms) : split_k;
+    g.items = (long)g.m_tiles * g.n_tiles * g.split_k;
+    const int avail = max_smem - kTileBarBytes - 1024;   // barrier block + alignment slack
+    int st = avail / tile_stage_bytes(g.mt);
+    if (st > kTileMaxStages) st = kTileMaxStages;
+    g.stages = st;
+    g.smem_bytes = kTileBarBytes + 1024 + st * tile_stage_bytes(g.mt);
+    // each CTA takes the SM's whole tensor memory: ask for enough shared memory that two never share an SM
+    if (g.smem_bytes < 120 * 1024) g.smem_bytes = 120 * 1024;
+    g.ctas = (int)(g.items < sms ? g.items : sms);
+    return g;
+}
+
+size_t tile_partial_bytes(const TileGeom& g) {
+    return g.split_k > 1 ? round256((size_t)g.items * g.mt * kTileCols * sizeof(float)) : 0;
+}
+
+// cuTensorMapEncodeTiled, resolved through the runtime so that libcuda is not a link dependency.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// Activations A [M, K] FP16 row-major as a 2-D tensor (k innermost), box = 64 k x mt rows, 128-byte
+// swizzle; rows past M read as zero.
+bool make_act_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mt) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileStageK, (cuuint32_t)mt};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(A), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Path taken when the caller does not force one: the tile kernel from M = 32 up.
+int resolve_path(int M, int path) {
+    if (path == W4A16_PATH_AUTO) return M >= 32 ? W4A16_PATH_TILE : W4A16_PATH_DECODE;
+    return path;
+}
 
 // FP32 partials of the two-kernel reduce used by the plain path: [split_k][M][N].
 size_t simple_partial_bytes(int M, int N, int split_k) {
@@ -173,6 +260,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
     int G = K / group;
     switch (resolve_path(M, path)) {
         case W4A16_PATH_DECODE: return choose_split_decode(M, N, G, sm_count_or_default());
+        case W4A16_PATH_TILE: return choose_split_tile(M, N, G, sm_count_or_default());
         default: return 1;
     }
 }
@@ -190,6 +278,8 @@ size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k) {
         int s = split_k == 0 ? choose_split_decode(M, N, K / group, sm_count_or_default()) : split_k;
         size_t simple = simple_partial_bytes(M, N, s);
         if (simple > need) need = simple;
+        TileGeom tg = tile_geom(M, N, K / group, split_k, sm_count_or_default(), 227 * 1024);
+        if (tile_partial_bytes(tg) > need) need = tile_partial_bytes(tg);
     }
     return need == 0 ? 0 : kWsHeaderBytes + need;
 }
@@ -265,7 +355,6 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     if (!d->is_sm100) return W4A16_ERR_ARCH;
 
     path = resolve_path(M, path);
-    if (path == W4A16_PATH_TILE) return W4A16_ERR_PATH;
     if (split_k > 65535) return W4A16_ERR_SPLITK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __half* Ah = reinterpret_cast<const __half*>(A);
@@ -289,6 +378,42 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
             if (cudaGetLastError() != cudaSuccess) return W4A16_ERR_CUDA;
         }
         return W4A16_OK;
+    }
+
+    if (path == W4A16_PATH_TILE) {
+        TileGeom g = tile_geom(M, N, G, split_k, d->sm_count, d->max_smem_optin);
+        if (g.stages < 2) return W4A16_ERR_PATH;
+        if (g.split_k > 1) {
+            if ((long)g.m_tiles * g.n_tiles * kTileDequantWarps > kMaxTickets) return W4A16_ERR_SPLITK;
+            if (ws_body_bytes < tile_partial_bytes(g)) return W4A16_ERR_WORKSPACE;
+        }
+        CUtensorMap tmap;
+        if (!make_act_tensor_map(&tmap, A, M, K, g.mt)) return W4A16_ERR_CUDA;
+        TileParams p;
+        p.Wq = static_cast<const uint32_t*>(Wq);
+        p.S = static_cast<const __half*>(S);
+        p.Z = static_cast<const uint32_t*>(Z);
+        p.C = Ch;
+        p.ws = reinterpret_cast<float*>(ws_body);
+        p.tickets = static_cast<int*>(d->ws);
+        p.M = M; p.N = N; p.K = K; p.G = G;
+        p.n_tiles = g.n_tiles;
+        p.m_tiles = g.m_tiles;
+        p.split_k = g.split_k;
+        p.stages = g.stages;
+        void (*kern)(const CUtensorMap, const TileParams) =
+            g.mt_index == 0 ? gemm_tile_kernel<32> : g.mt_index == 1 ? gemm_tile_kernel<64>
+            : g.mt_index == 2 ? gemm_tile_kernel<128> : gemm_tile_kernel<256>;
+        if (!d->tile_attr_set[g.mt_index]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return W4A16_ERR_CUDA;
+            }
+            d->tile_attr_set[g.mt_index] = true;
+        }
+        kern<<<dim3(g.ctas, 1, 1), kTileThreads, g.smem_bytes, st>>>(tmap, p);
+        return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
     }
 
     // W4A16_PATH_DECODE

@@ -10,26 +10,25 @@ namespace w4a16 {
 
 // ---------------------------------------------------------------------------------
 // Packed layout.  The weight matrix is cut into blocks of NT = 64 columns (n) by one
-// quantization group (128 k).  Block (t, g), t = n / 64, g = k / 128, G = K / 128:
+// quantization group (128 k).  Block (t, g), t = n / 64, g = k / 128, G = K / 128, sits at
+// position t*G + g of each packed buffer, so a K-slice of a column tile is one contiguous
+// byte range in each buffer (one TMA bulk copy each).
 //
-//   Wq  : 1024 uint32 (4 KiB) at word offset (t*G + g) * 1024, index
-//           ((c*4 + r)*32 + lane)*4 + j
-//         c = (k % 128) / 64  (64-wide k chunk), r = (n % 64) / 16 (16-row sub-tile),
-//         lane = gq*4 + tig (gq = 0..7, tig = 0..3), j = 0..3.
-//         The word holds 8 nibbles of rows n_lo = 64t + 16r + gq and n_hi = n_lo + 8 at
-//         k0 = 128g + 64c + 16 tig + 4j:
-//           nibble 0: (n_lo, k0)    nibble 4: (n_lo, k0+1)
-//           nibble 1: (n_hi, k0)    nibble 5: (n_hi, k0+1)
-//           nibble 2: (n_lo, k0+2)  nibble 6: (n_lo, k0+3)
-//           nibble 3: (n_hi, k0+2)  nibble 7: (n_hi, k0+3)
-//         so that one 128-bit load gives a lane 16 consecutive k of two rows, and the
-//         masks 0x000f000f / 0x00f000f0 on the word and on the word >> 8 give the four
-//         FP16x2 registers of an m16n8k16 A fragment (rows = n, columns = k).
-//   S   : 64 FP16 at element offset (t*G + g) * 64, index gq*8 + r*2 + h  (row 16r+gq+8h)
-//   Z   : 8 uint32 at word offset (t*G + g) * 8, word gq, nibble r*2 + h   (same row)
-//
-// All blocks of one column tile t are contiguous in g, so a K-slice of a tile is one
-// contiguous byte range in each of the three buffers (one TMA bulk copy each).
+//   Wq  : 1024 uint32 (4 KiB) per block.  Every word holds 8 consecutive k of ONE column n.
+//         The block is cut into 16 sub-blocks of 256 B: sub-block (c, rb), c = (k % 128) / 64,
+//         rb = (n % 64) / 8, at byte (c*8 + rb)*256, holds columns 8rb .. 8rb+7 (rho = n % 8)
+//         times 64 k as two 128-byte lines, line i = (k % 64) / 32.  Column rho's 16 bytes of
+//         line i (four words w = 0..3, k = 64c + 32i + 8w .. +7) sit at slot (rho + 4i) % 8 of
+//         the line.  With that rotation
+//           - eight threads that each own one column read their 16-byte chunk of a line from
+//             eight different slots (one 128-byte wavefront), and
+//           - a warp whose lane (gq = lane / 4, tig = lane % 4) reads 8 bytes of column gq at
+//             k = 16 tig .. 16 tig + 15 touches every bank once per half-warp.
+//         Inside a word, nibble p holds k offset 2 (p % 4) + p / 4, i.e. nibbles 0,4 = k+0,k+1;
+//         1,5 = k+2,k+3; 2,6 = k+4,k+5; 3,7 = k+6,k+7: the masks 0x000f000f / 0x00f000f0 on the
+//         word and on the word >> 8 then give four FP16x2 registers in ascending k.
+//   S   : 64 FP16 per block, element n % 64.
+//   Z   : 8 uint32 per block, word (n % 64) / 8, nibble n % 8.
 // ---------------------------------------------------------------------------------
 constexpr int kGroup = 128;
 constexpr int kTileN = 64;
@@ -37,6 +36,13 @@ constexpr int kBlockWords = 1024;  // uint32 per (tile, group) block of Wq
 constexpr int kBlockBytes = 4096;
 constexpr int kSBlockHalves = 64;
 constexpr int kZBlockWords = 8;
+
+// Word index inside a block of the word that holds column `col` (0..63) at k = 8*kw .. 8*kw+7
+// (kw = 0..15 inside the group).
+__host__ __device__ constexpr int block_word_index(int col, int kw) {
+    return ((kw >> 3) * 8 + (col >> 3)) * 64 + ((kw >> 2) & 1) * 32 + (((col & 7) + 4 * ((kw >> 2) & 1)) & 7) * 4 +
+           (kw & 3);
+}
 
 // Status word: a kernel whose bounded wait runs out ORs a code in here and returns.
 __device__ int g_status_word = 0;
@@ -117,11 +123,9 @@ constexpr uint32_t kMaskHi = 0x00f000f0u;
 constexpr uint32_t kMagic = 0x64006400u;  // FP16 1024.0 in both halves
 constexpr int kLutAndOr = (0xF0 & 0xCC) | 0xAA;  // (a & b) | c
 
-struct Frag4 {
-    __half2 lo_a;  // rows n_lo, k0,   k0+1   (A-fragment register a0)
-    __half2 hi_a;  // rows n_hi, k0,   k0+1   (a1)
-    __half2 lo_b;  // rows n_lo, k0+2, k0+3   (a2)
-    __half2 hi_b;  // rows n_hi, k0+2, k0+3   (a3)
+// Eight weights of one column, ascending k, as four FP16 pairs.
+struct Half8 {
+    __half2 h[4];  // h[j] = (k + 2j, k + 2j + 1)
 };
 
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t v) {
@@ -131,32 +135,30 @@ __device__ __forceinline__ uint32_t h2_as_u32(__half2 v) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// zlo = FP16x2 (1024 + z_lo) in both halves; zhi = FP16x2 -(64 + z_hi) in both halves.
+// zlo = FP16x2 (1024 + z) in both halves; zhi = FP16x2 -(64 + z) in both halves.
 __device__ __forceinline__ uint32_t zmagic_lo(uint32_t z) { return z * 0x00010001u + kMagic; }
 __device__ __forceinline__ uint32_t zmagic_hi(uint32_t z) { return z * 0x00100010u + 0xD400D400u; }
 
-// One packed word -> exact (q - z) as four FP16 pairs.
-__device__ __forceinline__ Frag4 unpack_word(uint32_t w, __half2 zlo, __half2 zhi) {
+// One packed word -> exact (q - z) for its eight k.
+__device__ __forceinline__ Half8 unpack_word(uint32_t w, __half2 zlo, __half2 zhi) {
     const __half2 sixteenth = __float2half2_rn(0.0625f);
-    Frag4 f;
-    uint32_t w8 = w >> 8;
-    f.lo_a = __hsub2(u32_as_h2(lop3<kLutAndOr>(w, kMaskLo, kMagic)), zlo);
-    f.hi_a = __hfma2(u32_as_h2(lop3<kLutAndOr>(w, kMaskHi, kMagic)), sixteenth, zhi);
-    f.lo_b = __hsub2(u32_as_h2(lop3<kLutAndOr>(w8, kMaskLo, kMagic)), zlo);
-    f.hi_b = __hfma2(u32_as_h2(lop3<kLutAndOr>(w8, kMaskHi, kMagic)), sixteenth, zhi);
+    Half8 f;
+    const uint32_t w8 = w >> 8;
+    f.h[0] = __hsub2(u32_as_h2(lop3<kLutAndOr>(w, kMaskLo, kMagic)), zlo);
+    f.h[1] = __hfma2(u32_as_h2(lop3<kLutAndOr>(w, kMaskHi, kMagic)), sixteenth, zhi);
+    f.h[2] = __hsub2(u32_as_h2(lop3<kLutAndOr>(w8, kMaskLo, kMagic)), zlo);
+    f.h[3] = __hfma2(u32_as_h2(lop3<kLutAndOr>(w8, kMaskHi, kMagic)), sixteenth, zhi);
     return f;
 }
 
-// One packed word -> four FP16 pairs of w16 = fp16_rn((q - z) * s): exact (q - z), then one
-// FP16 multiply by the row's scale (both halves of s_lo / s_hi hold the scale of n_lo / n_hi).
-// This is Algorithm 1's "Dequantize to FP16": the multiplicand of the GEMM is the FP16-rounded
-// weight, so every kernel that feeds tensor cores goes through here.
-__device__ __forceinline__ Frag4 dequant_word(uint32_t w, __half2 zlo, __half2 zhi, __half2 s_lo, __half2 s_hi) {
-    Frag4 f = unpack_word(w, zlo, zhi);
-    f.lo_a = __hmul2(f.lo_a, s_lo);
-    f.hi_a = __hmul2(f.hi_a, s_hi);
-    f.lo_b = __hmul2(f.lo_b, s_lo);
-    f.hi_b = __hmul2(f.hi_b, s_hi);
+// One packed word -> w16 = fp16_rn((q - z) * s) for its eight k: exact (q - z), then one FP16
+// multiply by the column's scale (both halves of s2).  This is Algorithm 1's "Dequantize to
+// FP16": the multiplicand of the GEMM is the FP16-rounded weight, so every kernel that feeds
+// tensor cores goes through here.
+__device__ __forceinline__ Half8 dequant_word(uint32_t w, __half2 zlo, __half2 zhi, __half2 s2) {
+    Half8 f = unpack_word(w, zlo, zhi);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) f.h[j] = __hmul2(f.h[j], s2);
     return f;
 }
 

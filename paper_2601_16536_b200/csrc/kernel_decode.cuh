@@ -10,10 +10,11 @@
 // A producer warp brings 4 units per stage (16 KiB of nibbles + their scales and zeros,
 // three TMA bulk copies) plus the matching activation rows into a shared-memory ring
 // guarded by mbarriers; stages never straddle a tile.  Eight consumer warps work on a
-// stage, two per unit, each on two of the block's four 16-row sub-tiles: a 128-bit shared
-// load gives a lane the A-fragment nibbles, a logic op and two FP16 ops per register turn
-// them into w16 = fp16_rn((q - z) s), and an m16n8k16 tensor-core MMA with the WEIGHTS as
-// the 16-row operand (MMA rows = n, MMA columns = batch rows) accumulates in FP32.
+// stage, two per unit, each on two of the block's four 16-column sub-tiles: two 64-bit shared
+// loads give a lane the nibbles of columns gq and gq + 8 at its 16 k, a logic op and two FP16
+// ops per register turn them into w16 = fp16_rn((q - z) s), and an m16n8k16 tensor-core MMA
+// with the WEIGHTS as the 16-row operand (MMA rows = n, MMA columns = batch rows) accumulates
+// in FP32.
 //
 // When a CTA leaves a tile it adds its warps' sums in a fixed order through shared
 // memory.  If it covered the tile's whole K range it writes FP16 C.  Otherwise it stores
@@ -64,13 +65,14 @@ __host__ __device__ inline int decode_smem_bytes(int mb, int stages) {
     return 128 + decode_red_bytes(mb) + stages * decode_stage_bytes(mb);
 }
 
-__device__ __forceinline__ void mma_m16n8k16(float (&d)[4], const Frag4& a, uint32_t b0, uint32_t b1) {
+// D += A . B with A = (a0: row gq, a1: row gq + 8, a2 / a3: the same rows, second k pair).
+__device__ __forceinline__ void mma_m16n8k16(float (&d)[4], __half2 a0, __half2 a1, __half2 a2, __half2 a3,
+                                             uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(h2_as_u32(a.lo_a)), "r"(h2_as_u32(a.hi_a)), "r"(h2_as_u32(a.lo_b)), "r"(h2_as_u32(a.hi_b)),
-          "r"(b0), "r"(b1));
+        : "r"(h2_as_u32(a0)), "r"(h2_as_u32(a1)), "r"(h2_as_u32(a2)), "r"(h2_as_u32(a3)), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ void consumer_bar() {
@@ -211,23 +213,26 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
             if (!mbar_wait(&full[slot], phase)) return;  // status recorded; every consumer warp sees it
             if (us < gc) {
                 const unsigned char* st = stage0 + (size_t)slot * stage_bytes;
-                const uint4* wsm = reinterpret_cast<const uint4*>(st + us * kBlockBytes);
+                const unsigned char* wst = st + us * kBlockBytes;
                 const unsigned char* a_s = st + kDecStageA + us * (kGroup * 2);
 
-                // scales / zero points of this lane's rows 16r + gq + 8h, r = r0, r0 + 1
-                const uint2 sraw = *reinterpret_cast<const uint2*>(st + kDecStageS + us * (kSBlockHalves * 2) +
-                                                                   gq * 16 + r0 * 4);
-                const uint32_t zw =
-                    *reinterpret_cast<const uint32_t*>(st + kDecStageZ + us * (kZBlockWords * 4) + gq * 4) >> (8 * r0);
-                const uint32_t sw[2] = {sraw.x, sraw.y};
-                __half2 s_lo[2], s_hi[2], zlo[2], zhi[2];
+                // scales / zero points of this lane's columns 16 rr + gq and 16 rr + gq + 8, rr = r0, r0 + 1
+                const __half* sp = reinterpret_cast<const __half*>(st + kDecStageS + us * (kSBlockHalves * 2));
+                const uint4 zq = *reinterpret_cast<const uint4*>(st + kDecStageZ + us * (kZBlockWords * 4) + r0 * 8);
+                const uint32_t zw[4] = {zq.x, zq.y, zq.z, zq.w};   // columns 8 (2 r0 + i) .. + 7
+                __half2 s_a[2], s_b[2], zlo_a[2], zhi_a[2], zlo_b[2], zhi_b[2];
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
-                    s_lo[r] = __half2half2(__low2half(u32_as_h2(sw[r])));   // row 16(r0+r) + gq
-                    s_hi[r] = __half2half2(__high2half(u32_as_h2(sw[r])));  // row 16(r0+r) + gq + 8
-                    zlo[r] = u32_as_h2(zmagic_lo((zw >> (8 * r)) & 15u));
-                    zhi[r] = u32_as_h2(zmagic_hi((zw >> (8 * r + 4)) & 15u));
+                    s_a[r] = __half2half2(sp[(r0 + r) * 16 + gq]);
+                    s_b[r] = __half2half2(sp[(r0 + r) * 16 + gq + 8]);
+                    const uint32_t za = (zw[2 * r] >> (4 * gq)) & 15u, zb = (zw[2 * r + 1] >> (4 * gq)) & 15u;
+                    zlo_a[r] = u32_as_h2(zmagic_lo(za));
+                    zhi_a[r] = u32_as_h2(zmagic_hi(za));
+                    zlo_b[r] = u32_as_h2(zmagic_lo(zb));
+                    zhi_b[r] = u32_as_h2(zmagic_hi(zb));
                 }
+                // this lane's 8 bytes of a column's 64-k line pair: k = 16 tig .. 16 tig + 15
+                const int woff = (tig >> 1) * 128 + ((gq + 4 * (tig >> 1)) & 7) * 16 + (tig & 1) * 8;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     // B fragments: batch row 8 mb + gq, 16 consecutive k per lane
@@ -242,14 +247,21 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
                     }
 #pragma unroll
                     for (int r = 0; r < 2; ++r) {
-                        const uint4 wv = wsm[(c * 4 + r0 + r) * 32 + lane];
-                        const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+                        const unsigned char* sub = wst + (c * 8 + 2 * (r0 + r)) * 256 + woff;
+                        const uint2 wa = *reinterpret_cast<const uint2*>(sub);        // column 16 rr + gq
+                        const uint2 wb = *reinterpret_cast<const uint2*>(sub + 256);  // column 16 rr + gq + 8
+                        const uint32_t wwa[2] = {wa.x, wa.y}, wwb[2] = {wb.x, wb.y};
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const Frag4 f = dequant_word(ww[j], zlo[r], zhi[r], s_lo[r], s_hi[r]);
+                        for (int wi = 0; wi < 2; ++wi) {
+                            const Half8 fa = dequant_word(wwa[wi], zlo_a[r], zhi_a[r], s_a[r]);
+                            const Half8 fb = dequant_word(wwb[wi], zlo_b[r], zhi_b[r], s_b[r]);
 #pragma unroll
-                            for (int mb = 0; mb < MB; ++mb)
-                                mma_m16n8k16(acc[r][mb], f, bw[mb][2 * j], bw[mb][2 * j + 1]);
+                            for (int mb = 0; mb < MB; ++mb) {
+                                mma_m16n8k16(acc[r][mb], fa.h[0], fb.h[0], fa.h[1], fb.h[1], bw[mb][4 * wi],
+                                             bw[mb][4 * wi + 1]);
+                                mma_m16n8k16(acc[r][mb], fa.h[2], fb.h[2], fa.h[3], fb.h[3], bw[mb][4 * wi + 2],
+                                             bw[mb][4 * wi + 3]);
+                            }
                         }
                     }
                 }

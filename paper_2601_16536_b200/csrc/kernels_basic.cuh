@@ -7,52 +7,56 @@
 namespace w4a16 {
 
 // ------------------------------------------------------------------ pack
-// One thread per packed word.  Pure bit moves (Section 2.2 storage packing).
+// Decode a packed word's position: idx -> block, column inside the tile, first k inside the group.
+__device__ __forceinline__ void word_position(size_t idx, size_t& blk, int& col, int& kw) {
+    const int within = (int)(idx & 1023);
+    blk = idx >> 10;
+    const int c = within >> 9, rb = (within >> 6) & 7, i = (within >> 5) & 1, slot = (within >> 2) & 7;
+    col = rb * 8 + ((slot - 4 * i) & 7);
+    kw = c * 8 + i * 4 + (within & 3);
+}
+
+// One thread per packed word.  Pure bit moves (Section 2.2 storage packing): the word's eight k
+// are one raw word of the same column; only the nibble order inside the word changes.
 __global__ void pack_wq_kernel(const uint32_t* __restrict__ raw, uint32_t* __restrict__ out, int N, int G,
                                size_t total_words) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total_words) return;
-    int j = (int)(idx & 3);
-    int lane = (int)((idx >> 2) & 31);
-    int r = (int)((idx >> 7) & 3);
-    int c = (int)((idx >> 9) & 1);
-    size_t blk = idx >> 10;
-    int t = (int)(blk / G), g = (int)(blk % G);
-    int tig = lane & 3, gq = lane >> 2;
-    int n_lo = t * kTileN + r * 16 + gq;
-    int k0 = g * kGroup + c * 64 + tig * 16 + j * 4;
-    int sh = (k0 & 7) * 4;  // 0 or 16: the four k sit in one half of a raw word
-    uint32_t a = (raw[(size_t)(k0 >> 3) * N + n_lo] >> sh) & 0xFFFFu;
-    uint32_t b = (raw[(size_t)(k0 >> 3) * N + n_lo + 8] >> sh) & 0xFFFFu;
-    uint32_t a0 = a & 15u, a1 = (a >> 4) & 15u, a2 = (a >> 8) & 15u, a3 = (a >> 12) & 15u;
-    uint32_t b0 = b & 15u, b1 = (b >> 4) & 15u, b2 = (b >> 8) & 15u, b3 = (b >> 12) & 15u;
-    out[idx] = a0 | (b0 << 4) | (a2 << 8) | (b2 << 12) | (a1 << 16) | (b1 << 20) | (a3 << 24) | (b3 << 28);
+    size_t blk;
+    int col, kw;
+    word_position(idx, blk, col, kw);
+    const int t = (int)(blk / G), g = (int)(blk % G);
+    const uint32_t r = raw[(size_t)(g * (kGroup / 8) + kw) * N + (size_t)t * kTileN + col];
+    uint32_t w = 0;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        const int off = 2 * (p & 3) + (p >> 2);  // k offset held by nibble p
+        w |= ((r >> (4 * off)) & 15u) << (4 * p);
+    }
+    out[idx] = w;
 }
 
 __global__ void pack_s_kernel(const uint16_t* __restrict__ raw, uint16_t* __restrict__ out, int N, int G,
                               size_t total) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
-    int e = (int)(idx & 63);
-    size_t blk = idx >> 6;
-    int t = (int)(blk / G), g = (int)(blk % G);
-    int gq = e >> 3, r = (e >> 1) & 3, h = e & 1;
-    out[idx] = raw[(size_t)g * N + t * kTileN + r * 16 + gq + 8 * h];
+    const int col = (int)(idx & 63);
+    const size_t blk = idx >> 6;
+    const int t = (int)(blk / G), g = (int)(blk % G);
+    out[idx] = raw[(size_t)g * N + (size_t)t * kTileN + col];
 }
 
 __global__ void pack_z_kernel(const uint8_t* __restrict__ raw, uint32_t* __restrict__ out, int N, int G,
                               size_t total_words) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total_words) return;
-    int gq = (int)(idx & 7);
-    size_t blk = idx >> 3;
-    int t = (int)(blk / G), g = (int)(blk % G);
+    const int rb = (int)(idx & 7);
+    const size_t blk = idx >> 3;
+    const int t = (int)(blk / G), g = (int)(blk % G);
     uint32_t w = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        int r = i >> 1, h = i & 1;
-        w |= (uint32_t)(raw[(size_t)g * N + t * kTileN + r * 16 + gq + 8 * h] & 15u) << (4 * i);
-    }
+    for (int i = 0; i < 8; ++i)
+        w |= (uint32_t)(raw[(size_t)g * N + (size_t)t * kTileN + rb * 8 + i] & 15u) << (4 * i);
     out[idx] = w;
 }
 
@@ -65,38 +69,24 @@ __global__ void dequant_kernel(const uint32_t* __restrict__ Wq, const __half* __
                                size_t total_words) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total_words) return;
-    int j = (int)(idx & 3);
-    int lane = (int)((idx >> 2) & 31);
-    int r = (int)((idx >> 7) & 3);
-    int c = (int)((idx >> 9) & 1);
-    size_t blk = idx >> 10;
-    int t = (int)(blk / G), g = (int)(blk % G);
-    int tig = lane & 3, gq = lane >> 2;
-    int n_lo = t * kTileN + r * 16 + gq;
-    int k0 = g * kGroup + c * 64 + tig * 16 + j * 4;
-
-    uint32_t zw = Z[blk * kZBlockWords + gq];
-    __half2 zlo = u32_as_h2(zmagic_lo((zw >> (8 * r)) & 15u));
-    __half2 zhi = u32_as_h2(zmagic_hi((zw >> (8 * r + 4)) & 15u));
-    __half s_lo = S[blk * kSBlockHalves + gq * 8 + r * 2];
-    __half s_hi = S[blk * kSBlockHalves + gq * 8 + r * 2 + 1];
-
-    const Frag4 f = dequant_word(Wq[idx], zlo, zhi, __half2half2(s_lo), __half2half2(s_hi));
-    const __half2 wa = f.lo_a, wb = f.lo_b, wc = f.hi_a, wd = f.hi_b;
-    __half* p = W16 + (size_t)k0 * N + n_lo;
-    p[0] = __low2half(wa);
-    p[(size_t)N] = __high2half(wa);
-    p[(size_t)2 * N] = __low2half(wb);
-    p[(size_t)3 * N] = __high2half(wb);
-    p[8] = __low2half(wc);
-    p[(size_t)N + 8] = __high2half(wc);
-    p[(size_t)2 * N + 8] = __low2half(wd);
-    p[(size_t)3 * N + 8] = __high2half(wd);
+    size_t blk;
+    int col, kw;
+    word_position(idx, blk, col, kw);
+    const int t = (int)(blk / G), g = (int)(blk % G);
+    const uint32_t z = (Z[blk * kZBlockWords + (col >> 3)] >> (4 * (col & 7))) & 15u;
+    const __half s = S[blk * kSBlockHalves + col];
+    const Half8 f = dequant_word(Wq[idx], u32_as_h2(zmagic_lo(z)), u32_as_h2(zmagic_hi(z)), __half2half2(s));
+    __half* p = W16 + (size_t)(g * kGroup + kw * 8) * N + (size_t)t * kTileN + col;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        p[(size_t)(2 * j) * N] = __low2half(f.h[j]);
+        p[(size_t)(2 * j + 1) * N] = __high2half(f.h[j]);
+    }
 }
 
 // ------------------------------------------------------------------ plain GEMM
 // Correct-first kernel: one thread per output column of a 64-column tile, kSimpleMB batch
-// rows per thread, FP32 FMA in ascending k over this CTA's K-slice.  Grid: (N/64,
+// rows per thread, FP32 FMA over this CTA's K-slice.  Grid: (N/64,
 // ceil(M/kSimpleMB), split_k).  With split_k == 1 it writes FP16 C, else FP32 partials
 // ws[split][M][N] (Algorithm 1, Phase 2) for splitk_reduce_kernel.
 constexpr int kSimpleMB = 4;
@@ -111,9 +101,8 @@ __global__ void __launch_bounds__(64)
 gemm_simple_kernel(const __half* __restrict__ A, const uint32_t* __restrict__ Wq, const __half* __restrict__ S,
                    const uint32_t* __restrict__ Z, __half* __restrict__ C, float* __restrict__ ws, int M, int N,
                    int K, int G, int split_k) {
-    int t = blockIdx.x, m0 = blockIdx.y * kSimpleMB, sp = blockIdx.z;
-    int e = threadIdx.x;  // row inside the tile
-    int r = e >> 4, gq = e & 7, h = (e >> 3) & 1;
+    const int t = blockIdx.x, m0 = blockIdx.y * kSimpleMB, sp = blockIdx.z;
+    const int col = threadIdx.x;  // column inside the tile
     int g0, ng;
     slice_of(G, split_k, sp, g0, ng);
 
@@ -122,30 +111,27 @@ gemm_simple_kernel(const __half* __restrict__ A, const uint32_t* __restrict__ Wq
     for (int i = 0; i < kSimpleMB; ++i) acc[i] = 0.f;
 
     for (int g = g0; g < g0 + ng; ++g) {
-        size_t blk = (size_t)t * G + g;
-        int z = (int)((Z[blk * kZBlockWords + gq] >> (4 * (r * 2 + h))) & 15u);
-        float s = __half2float(S[blk * kSBlockHalves + gq * 8 + r * 2 + h]);
+        const size_t blk = (size_t)t * G + g;
+        const int z = (int)((Z[blk * kZBlockWords + (col >> 3)] >> (4 * (col & 7))) & 15u);
+        const float s = __half2float(S[blk * kSBlockHalves + col]);
         const uint32_t* wb = Wq + blk * kBlockWords;
-        for (int c = 0; c < 2; ++c)
-            for (int tig = 0; tig < 4; ++tig)
-                for (int j = 0; j < 4; ++j) {
-                    uint32_t w = wb[((c * 4 + r) * 32 + gq * 4 + tig) * 4 + j] >> (4 * h);
-                    int k0 = g * kGroup + c * 64 + tig * 16 + j * 4;
-                    // nibbles (after the shift by 4h): 0 -> k0, 4 -> k0+1, 2 -> k0+2, 6 -> k0+3
-                    int q[4] = {(int)(w & 15u), (int)((w >> 16) & 15u), (int)((w >> 8) & 15u),
-                                (int)((w >> 24) & 15u)};
+        for (int kw = 0; kw < kGroup / 8; ++kw) {
+            const uint32_t w = wb[block_word_index(col, kw)];
+            const int k0 = g * kGroup + kw * 8;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float w16 = __half2float(__float2half_rn((float)(q[i] - z) * s));
+            for (int p = 0; p < 8; ++p) {
+                const int off = 2 * (p & 3) + (p >> 2);
+                const int q = (int)((w >> (4 * p)) & 15u);
+                const float w16 = __half2float(__float2half_rn((float)(q - z) * s));
 #pragma unroll
-                        for (int mm = 0; mm < kSimpleMB; ++mm) {
-                            if (m0 + mm < M)
-                                acc[mm] = fmaf(__half2float(A[(size_t)(m0 + mm) * K + k0 + i]), w16, acc[mm]);
-                        }
-                    }
+                for (int mm = 0; mm < kSimpleMB; ++mm) {
+                    if (m0 + mm < M)
+                        acc[mm] = fmaf(__half2float(A[(size_t)(m0 + mm) * K + k0 + off]), w16, acc[mm]);
                 }
+            }
+        }
     }
-    int n = t * kTileN + r * 16 + gq + 8 * h;
+    const int n = t * kTileN + col;
 #pragma unroll
     for (int mm = 0; mm < kSimpleMB; ++mm) {
         if (m0 + mm < M) {
