@@ -379,15 +379,19 @@ def run_ours(args):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        t0 = time.perf_counter()
-        worst = 0.0
+        worst, reps_cpu, dt = 0.0, 0, 0.0
+        while dt < 10.0 and reps_cpu < 64:     # whole steps until about 10 s of CPU work
+            t0 = time.perf_counter()
+            refs = [oracle.gemm(acts_np[i], layer.raw["Wq"], layer.raw["S"], layer.raw["Z"], M, N, K, 128)
+                    for i, M in enumerate(SWEEP_M)]
+            dt += time.perf_counter() - t0
+            reps_cpu += 1
         for i, M in enumerate(SWEEP_M):
-            ref = oracle.gemm(acts_np[i], layer.raw["Wq"], layer.raw["S"], layer.raw["Z"], M, N, K, 128)
             got = outs[i].cpu().numpy().astype(np.float64)   # result of the last timed call
-            worst = max(worst, float(np.max(np.abs(got - ref) / (1.0 + np.abs(ref)))))
-        dt = time.perf_counter() - t0
-        cpu = {"value": step_bytes / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": "one full step (all 5 GEMMs, all columns), %.1f s" % dt,
+            worst = max(worst, float(np.max(np.abs(got - refs[i]) / (1.0 + np.abs(refs[i])))))
+        cpu = {"value": step_bytes * reps_cpu / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(),
+               "kind": "oracle",
+               "sample": "%d full steps (all 5 GEMMs, all columns), %.1f s of CPU time" % (reps_cpu, dt),
                "max_elem_err_vs_gpu": worst}
 
     if rank == 0:
@@ -442,9 +446,16 @@ def run_one(args):
     assert B.w4a16_device_status() == 0
     us = e0.elapsed_time(e1) * 1e3 / args.calls
     byts = wl.algorithmic_bytes(M, K, N)
-    print(json.dumps({"one": [M, K, N], "path": args.path, "split_k": args.split_k, "calls": args.calls,
-                      "us_per_call_stream": us, "eff_GBps": byts / us / 1e3,
-                      "tflops": 2.0 * M * N * K / us / 1e6, "copies": layer.copies}))
+    out = {"one": [M, K, N], "path": args.path, "split_k": args.split_k, "calls": args.calls,
+           "us_per_call_stream": us, "copies": layer.copies}
+    if args.graph:
+        # the same call inside replayed CUDA graphs: device time of back-to-back launches
+        g_us = _time_calls(lambda: B.w4a16_gemm(A, layer.take(), C, split_k=args.split_k, path=args.path),
+                           3, max(args.calls, 64), torch, per_graph=min(32, max(2, layer.copies))) * 1e6
+        hbm_peak, tc_peak, _ = _peaks()
+        out.update(us_per_call_graph=g_us, eff_GBps=byts / g_us / 1e3, tflops=2.0 * M * N * K / g_us / 1e6,
+                   roofline_frac=max(byts / (hbm_peak * 1e3), 2.0 * M * N * K / (tc_peak * 1e6)) / g_us)
+    print(json.dumps(out))
     del ws
 
 
@@ -464,6 +475,7 @@ def main():
     ap.add_argument("--one", type=lambda s: [int(x) for x in s.split(",")], default=None,
                     help="M,K,N: time this one shape with plain stream launches and exit")
     ap.add_argument("--calls", type=int, default=20, help="launches of --one")
+    ap.add_argument("--graph", action="store_true", help="--one: also time the call inside CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="kernel path of --one (0 auto, 1 simple, 2 decode, 3 tile)")
     ap.add_argument("--rotation-mb", type=int, default=512, help="bytes of rotating weight copies of --one")
     args = ap.parse_args()

@@ -63,7 +63,7 @@ enum {
     W4A16_PATH_SIMPLE = 1, /* plain FP32-FMA kernel, any M; two-kernel Split-K reduce */
     W4A16_PATH_DECODE = 2, /* small-M bandwidth-bound kernel (M <= 64): TMA bulk staging,
                               in-register unpack, warp-level tensor-core MMA */
-    W4A16_PATH_TILE = 3    /* tcgen05 / TMEM tile kernel for large M */
+    W4A16_PATH_TILE = 3    /* tcgen05 / TMEM tile kernel, any M (batch tiles of 16 .. 256 rows) */
 };
 
 const char *w4a16_strerror(int code);
@@ -81,10 +81,11 @@ size_t w4a16_packed_z_bytes(int N, int K, int group);
  * workspace is needed.
  * w4a16_set_workspace: registers the buffer for the CURRENT device (one per device, per
  * process; replaces the previous one; dev_ptr == NULL, bytes == 0 unregisters).  The
- * buffer must be 256-byte aligned, stays owned by the caller and must outlive every gemm
- * call enqueued while it is registered.  The call zeroes the buffer's first 16 KiB on the
- * default stream and waits for that.  gemm calls that need the workspace and overlap on
+ * buffer must be 256-byte aligned and at least W4A16_WORKSPACE_HEADER_BYTES long, stays
+ * owned by the caller and must outlive every gemm call enqueued while it is registered.  The
+ * call zeroes that header (the kernels' ticket counters) on the default stream and waits.  gemm calls that need the workspace and overlap on
  * the GPU (different streams) race on it; serialise them or use split_k = 1. */
+#define W4A16_WORKSPACE_HEADER_BYTES (16384u + 131072u)
 size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k);
 int w4a16_set_workspace(void *dev_ptr, size_t bytes);
 
@@ -116,7 +117,11 @@ int w4a16_dequant(const void *Wq, const void *S, const void *Z, uint16_t *W16,
  *   split_k   0 = automatic, else 1 <= split_k <= K/group (some paths cap it lower and
  *             return W4A16_ERR_SPLITK beyond their cap)
  * Results are bit-identical from run to run for fixed arguments.  If the chosen
- * split needs workspace and too little is registered: W4A16_ERR_WORKSPACE. */
+ * split needs workspace and too little is registered: W4A16_ERR_WORKSPACE.
+ * Ordering: A, C and the workspace are touched in stream order.  The packed buffers Wq, S, Z
+ * may be read (prefetched) while the previous kernel of the stream is still running, so
+ * they must not be written by in-flight work other than a w4a16_pack enqueued earlier on the
+ * same device (the library orders the next GEMM launch after it); pack weights once, at load. */
 int w4a16_gemm(const uint16_t *A, const void *Wq, const void *S, const void *Z, uint16_t *C,
                int M, int N, int K, int group, int split_k, w4a16_stream_t stream);
 

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libw4a16.so")
 
 PATH_AUTO, PATH_SIMPLE, PATH_DECODE, PATH_TILE = 0, 1, 2, 3
 GROUP = 128
+WS_HEADER_BYTES = 16384 + 131072   # W4A16_WORKSPACE_HEADER_BYTES
 
 EXPORTS = (
     "w4a16_strerror", "w4a16_packed_wq_bytes", "w4a16_packed_s_bytes", "w4a16_packed_z_bytes",
@@ -203,9 +204,9 @@ def w4a16_gemm_static_ws(A: torch.Tensor, pw: PackedWeights, C: Optional[torch.T
 def ensure_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     """Allocate (with torch) and register a workspace of at least ``nbytes``; returns the tensor,
     which the caller must keep alive while it is registered."""
-    ws = torch.empty(max(int(nbytes), 16384) + 256, dtype=torch.uint8, device=device)
+    ws = torch.empty(max(int(nbytes), WS_HEADER_BYTES) + 256, dtype=torch.uint8, device=device)
     off = (-ws.data_ptr()) % 256
-    view = ws[off:off + max(int(nbytes), 16384)]
+    view = ws[off:off + max(int(nbytes), WS_HEADER_BYTES)]
     w4a16_set_workspace(view)
     view._keepalive = ws  # type: ignore[attr-defined]
     return view

@@ -26,7 +26,12 @@ struct DeviceState {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     bool decode_attr_set[3] = {false, false, false};
-    bool tile_attr_set[4] = {false, false, false, false};
+    bool tile_attr_set[5] = {false, false, false, false, false};
+    // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
+    // kernel in its stream has finished.  After w4a16_pack was enqueued the next GEMM launch is
+    // therefore a plain, fully ordered one (it runs after the pack kernels), and only the launches
+    // after it overlap their predecessor again.
+    bool pdl_ok = false;
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -116,42 +121,41 @@ int choose_split_decode(int M, int N, int G, int sms) {
 }
 
 // ---- tile-path launch geometry ----------------------------------------------------
-// MT (batch rows per CTA tile = UMMA N) is the smallest of 32, 64, 128, 256 that covers M, else 256.
+// MT (batch rows per CTA tile = UMMA N) is the smallest of 16, 32, 64, 128, 256 that covers M, else
+// 256.  The unit range (batch tile x column tile x group) is cut into `nchunks` chunks for `ctas`
+// persistent CTAs: balanced chunks, one per CTA, when the caller leaves split_k open; S slices
+// per tile otherwise.
 struct TileGeom {
-    int mt, mt_index, m_tiles, n_tiles, split_k, stages, smem_bytes, ctas;
-    long items;
+    int mt, mt_index, m_tiles, n_tiles, split_k, nchunks, stages, smem_bytes, ctas;
+    long tiles;
 };
 
-int tile_mt_index(int M) { return M <= 32 ? 0 : M <= 64 ? 1 : M <= 128 ? 2 : 3; }
+constexpr size_t kTileTicketBytes = 131072;   // 16 counters per tile, after the 16 KiB of the small-M kernel
+constexpr size_t kWsFullHeaderBytes = kWsHeaderBytes + kTileTicketBytes;
+constexpr long kTileMaxTicketTiles = kTileTicketBytes / (sizeof(int) * kTileDequantWarps);
 
-// Split factor of the tile path when the caller leaves it open (the paper takes S as an input).
-// Cost model: the grid runs ceil(tiles * S / SMs) waves, each as long as one item: ceil(G / S)
-// groups of main loop plus a fixed part (pipeline fill, epilogue, partial-tile exchange) worth
-// about six groups.  Slices keep at least four groups; S <= 16; S = 1 once the tiles fill the SMs.
-int choose_split_tile(int M, int N, int G, int sms) {
-    const int mt = 32 << tile_mt_index(M);
-    const long tiles = (long)((N + kTileCols - 1) / kTileCols) * ((M + mt - 1) / mt);
-    int best = 1;
-    long best_cost = -1;
-    for (int s = 1; s <= 16 && (s == 1 || G / s >= 4); ++s) {
-        const long waves = (tiles * s + sms - 1) / sms;
-        const long cost = waves * ((G + s - 1) / s + (s > 1 ? 6 : 4));
-        if (best_cost < 0 || cost < best_cost) {
-            best_cost = cost;
-            best = s;
-        }
-    }
-    return best;
-}
+int tile_mt_index(int M) { return M <= 16 ? 0 : M <= 32 ? 1 : M <= 64 ? 2 : M <= 128 ? 3 : 4; }
 
 TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     TileGeom g;
     g.mt_index = tile_mt_index(M);
-    g.mt = 32 << g.mt_index;
+    g.mt = 16 << g.mt_index;
     g.m_tiles = (M + g.mt - 1) / g.mt;
     g.n_tiles = (N + kTileCols - 1) / kTileCols;
-    g.split_k = split_k == 0 ? choose_split_tile(M, N, G, sms) : split_k;
-    g.items = (long)g.m_tiles * g.n_tiles * g.split_k;
+    g.tiles = (long)g.m_tiles * g.n_tiles;
+    // more tiles than ticket counters: whole tiles only (no partial tiles, no tickets)
+    if (split_k == 0 && g.tiles > kTileMaxTicketTiles) split_k = 1;
+    g.split_k = split_k;
+    if (split_k == 0) {
+        const long units = g.tiles * G;
+        long n = units / 2;                      // at least two units (four stages) per chunk
+        if (n < 1) n = 1;
+        if (n > sms) n = sms;
+        g.nchunks = (int)n;
+    } else {
+        g.nchunks = (int)(g.tiles * split_k);
+    }
+    g.ctas = g.nchunks < sms ? g.nchunks : sms;
     const int avail = max_smem - kTileBarBytes - 1024;   // barrier block + alignment slack
     int st = avail / tile_stage_bytes(g.mt);
     if (st > kTileMaxStages) st = kTileMaxStages;
@@ -159,12 +163,23 @@ TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     g.smem_bytes = kTileBarBytes + 1024 + st * tile_stage_bytes(g.mt);
     // each CTA takes the SM's whole tensor memory: ask for enough shared memory that two never share an SM
     if (g.smem_bytes < 120 * 1024) g.smem_bytes = 120 * 1024;
-    g.ctas = (int)(g.items < sms ? g.items : sms);
     return g;
 }
 
-size_t tile_partial_bytes(const TileGeom& g) {
-    return g.split_k > 1 ? round256((size_t)g.items * g.mt * kTileCols * sizeof(float)) : 0;
+// Partial-tile slots of the tile path: two per chunk.  Nothing when every chunk is a whole tile.
+size_t tile_workspace_bytes(const TileGeom& g) {
+    if (g.split_k == 1) return 0;
+    return round256((size_t)2 * g.nchunks * g.mt * kTileCols * sizeof(float));
+}
+
+// Nominal split factor of the tile path's schedule: how many chunks share one tile's K range.
+int choose_split_tile(int M, int N, int G, int sms) {
+    TileGeom g = tile_geom(M, N, G, 0, sms, 227 * 1024);
+    if (g.split_k == 1) return 1;
+    long s = (g.nchunks + g.tiles - 1) / g.tiles;
+    if (s < 1) s = 1;
+    if (s > G) s = G;
+    return (int)s;
 }
 
 // cuTensorMapEncodeTiled, resolved through the runtime so that libcuda is not a link dependency.
@@ -279,9 +294,9 @@ size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k) {
         size_t simple = simple_partial_bytes(M, N, s);
         if (simple > need) need = simple;
         TileGeom tg = tile_geom(M, N, K / group, split_k, sm_count_or_default(), 227 * 1024);
-        if (tile_partial_bytes(tg) > need) need = tile_partial_bytes(tg);
+        if (tile_workspace_bytes(tg) > need) need = tile_workspace_bytes(tg);
     }
-    return need == 0 ? 0 : kWsHeaderBytes + need;
+    return need == 0 ? 0 : kWsFullHeaderBytes + need;
 }
 
 int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
@@ -294,8 +309,9 @@ int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
         return W4A16_OK;
     }
     if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return W4A16_ERR_ALIGN;
-    if (bytes < kWsHeaderBytes) return W4A16_ERR_WORKSPACE;
-    if (cudaMemset(dev_ptr, 0, kWsHeaderBytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    if (bytes < kWsFullHeaderBytes) return W4A16_ERR_WORKSPACE;
+    // both kernels' ticket blocks start at zero (and leave zeros behind after every call)
+    if (cudaMemset(dev_ptr, 0, kWsFullHeaderBytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
         return W4A16_ERR_CUDA;
     }
@@ -321,6 +337,7 @@ int w4a16_pack(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_r
     pack_wq_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(Wq_raw, static_cast<uint32_t*>(Wq), N, G, words);
     pack_s_kernel<<<(unsigned)((sc + 255) / 256), 256, 0, st>>>(S_raw, static_cast<uint16_t*>(S), N, G, sc);
     pack_z_kernel<<<(unsigned)((zw + 255) / 256), 256, 0, st>>>(Z_raw, static_cast<uint32_t*>(Z), N, G, zw);
+    d->pdl_ok = false;
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
@@ -359,8 +376,9 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __half* Ah = reinterpret_cast<const __half*>(A);
     __half* Ch = reinterpret_cast<__half*>(C);
-    unsigned char* ws_body = d->ws ? static_cast<unsigned char*>(d->ws) + kWsHeaderBytes : nullptr;
-    const size_t ws_body_bytes = d->ws_bytes > kWsHeaderBytes ? d->ws_bytes - kWsHeaderBytes : 0;
+    // registered workspace: [16 KiB small-M tickets][128 KiB tile tickets][partial results]
+    unsigned char* ws_body = d->ws ? static_cast<unsigned char*>(d->ws) + kWsFullHeaderBytes : nullptr;
+    const size_t ws_body_bytes = d->ws_bytes > kWsFullHeaderBytes ? d->ws_bytes - kWsFullHeaderBytes : 0;
 
     if (path == W4A16_PATH_SIMPLE) {
         if (split_k == 0) split_k = choose_split_decode(M, N, G, d->sm_count);
@@ -383,9 +401,9 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     if (path == W4A16_PATH_TILE) {
         TileGeom g = tile_geom(M, N, G, split_k, d->sm_count, d->max_smem_optin);
         if (g.stages < 2) return W4A16_ERR_PATH;
-        if (g.split_k > 1) {
-            if ((long)g.m_tiles * g.n_tiles * kTileDequantWarps > kMaxTickets) return W4A16_ERR_SPLITK;
-            if (ws_body_bytes < tile_partial_bytes(g)) return W4A16_ERR_WORKSPACE;
+        if (g.split_k != 1) {
+            if (g.tiles > kTileMaxTicketTiles) return W4A16_ERR_SPLITK;
+            if (ws_body_bytes < tile_workspace_bytes(g)) return W4A16_ERR_WORKSPACE;
         }
         CUtensorMap tmap;
         if (!make_act_tensor_map(&tmap, A, M, K, g.mt)) return W4A16_ERR_CUDA;
@@ -394,16 +412,18 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
         p.S = static_cast<const __half*>(S);
         p.Z = static_cast<const uint32_t*>(Z);
         p.C = Ch;
+        p.tickets = reinterpret_cast<int*>(d->ws ? static_cast<unsigned char*>(d->ws) + kWsHeaderBytes : nullptr);
         p.ws = reinterpret_cast<float*>(ws_body);
-        p.tickets = static_cast<int*>(d->ws);
         p.M = M; p.N = N; p.K = K; p.G = G;
         p.n_tiles = g.n_tiles;
         p.m_tiles = g.m_tiles;
         p.split_k = g.split_k;
+        p.nchunks = g.nchunks;
         p.stages = g.stages;
         void (*kern)(const CUtensorMap, const TileParams) =
-            g.mt_index == 0 ? gemm_tile_kernel<32> : g.mt_index == 1 ? gemm_tile_kernel<64>
-            : g.mt_index == 2 ? gemm_tile_kernel<128> : gemm_tile_kernel<256>;
+            g.mt_index == 0 ? gemm_tile_kernel<16> : g.mt_index == 1 ? gemm_tile_kernel<32>
+            : g.mt_index == 2 ? gemm_tile_kernel<64> : g.mt_index == 3 ? gemm_tile_kernel<128>
+                                                                        : gemm_tile_kernel<256>;
         if (!d->tile_attr_set[g.mt_index]) {
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
                 cudaSuccess) {
@@ -412,8 +432,24 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
             }
             d->tile_attr_set[g.mt_index] = true;
         }
-        kern<<<dim3(g.ctas, 1, 1), kTileThreads, g.smem_bytes, st>>>(tmap, p);
-        return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
+        // programmatic dependent launch: this kernel's prologue and weight prefetch may overlap the
+        // tail of the previous kernel in the stream; it orders itself with griddepcontrol.wait
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(g.ctas, 1, 1);
+        cfg.blockDim = dim3(kTileThreads, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = d->pdl_ok ? 1 : 0;
+        d->pdl_ok = true;
+        if (cudaLaunchKernelEx(&cfg, kern, tmap, p) != cudaSuccess) {
+            cudaGetLastError();
+            return W4A16_ERR_CUDA;
+        }
+        return W4A16_OK;
     }
 
     // W4A16_PATH_DECODE

@@ -13,12 +13,28 @@
 // so dequantized weights never touch shared or global memory (Algorithm 1's Phase 1 output
 // stays on chip), and the activation tile is re-used by all 128 columns of the CTA tile.
 //
-// A work item is (column tile of 128 n, batch tile of MT m, K slice of whole groups); items are
-// dealt round-robin to a persistent grid.  One pipeline stage is 64 k: 4 KiB of nibbles, the
-// group's scales and zeros, and an MT x 64 FP16 activation box.  The two sets of four dequant
-// warps take alternate stages; inside a set warp w owns TMEM lanes 32 (w % 4) .. + 31, one
-// column n per thread.  All waits are bounded mbarrier waits; a wait that runs out records a
-// status code and the CTA drains and exits (TMEM is always released).
+// Work is counted in units: one unit = 128 columns x one group (128 k) of one batch tile, numbered
+// U = (batch tile * NT + column tile) * G + group.  The unit range is cut into chunks, each CTA of
+// the persistent grid walks its chunk(s) front to back:
+//   - balanced (split_k == 0): as many chunks as CTAs, equal to within one unit; a chunk may start
+//     and end inside a tile's K range and may cover several whole tiles in between;
+//   - classic Split-K (split_k = S): every tile's K range is cut into S slices of whole groups
+//     (Algorithm 1, Phase 2), chunks dealt round-robin.
+// The part of a chunk inside one tile is a segment: the accumulator is zeroed at its first MMA and
+// drained after its last.  A segment that covers a whole tile is cast to FP16 and stored; any other
+// segment leaves as an FP32 partial tile in the workspace, and the warp that draws the last ticket
+// of its 32-column x MT/4-row region adds the partial regions in ascending K order (Phase 3).
+// No warp ever waits for another CTA, and the order of the sum is fixed, so results are
+// bit-identical from run to run.
+//
+// One pipeline stage is 64 k: 4 KiB of nibbles, the group's scales and zeros, and an MT x 64 FP16
+// activation box.  Four sets of four dequant warps take stages round-robin; inside a set warp w
+// owns TMEM lanes 32 (w % 4) .. + 31, one column n per thread.  With MT <= 128 two accumulators
+// alternate between segments, so one drains while the next fills.  The packed weights do not
+// depend on the previous kernel in the stream: under programmatic dependent launch the producer
+// fills the whole ring with them before griddepcontrol.wait, and only activations, C and the
+// workspace are touched after it.  All waits are bounded mbarrier waits; a wait that runs out
+// records a status code and the CTA drains and exits (TMEM is always released).
 #pragma once
 
 #include <cuda.h>
@@ -29,15 +45,16 @@ namespace w4a16 {
 
 constexpr int kTileCols = 128;                      // n per CTA tile = UMMA M
 constexpr int kTileStageK = 64;                     // k per pipeline stage
-constexpr int kTileDequantWarps = 8;
-constexpr int kTileThreads = (2 + kTileDequantWarps) * 32;   // producer, MMA, 8 dequant/epilogue warps
+constexpr int kTileDequantWarps = 16;               // four sets of four (one warp per TMEM lane quarter)
+constexpr int kTileSets = kTileDequantWarps / 4;
+constexpr int kTileThreads = (2 + kTileDequantWarps) * 32;   // producer, MMA, dequant/epilogue warps
 constexpr int kTileASlots = 8;                      // TMEM ring of A-operand slots (32 columns each)
-constexpr int kTileAColBase = 256;                  // D occupies columns [0, MT), the ring [256, 512)
+constexpr int kTileAColBase = 256;                  // accumulators in columns [0, 256), the ring in [256, 512)
 constexpr int kTileStageW = 0;                      // 2 x 2 KiB of nibbles (two 64-column packed tiles)
 constexpr int kTileStageS = 4096;                   // 2 x 64 FP16
 constexpr int kTileStageZ = 4352;                   // 2 x 8 uint32
 constexpr int kTileStageAct = 5120;                 // MT x 128 B, 1024-byte aligned (128B swizzle atom)
-constexpr int kTileMaxStages = 8;
+constexpr int kTileMaxStages = 16;
 constexpr int kTileBarBytes = 1024;
 
 __host__ __device__ constexpr int tile_stage_bytes(int mt) { return kTileStageAct + mt * 128; }
@@ -47,12 +64,13 @@ struct TileParams {
     const __half* S;
     const uint32_t* Z;
     __half* C;
-    float* ws;       // Split-K partial tiles [item][MT][128] FP32
-    int* tickets;    // zeroed counters, eight (one per epilogue warp) per (column tile, batch tile)
+    float* ws;       // partial tiles: [2 * nchunks slots][MT][128] FP32
+    int* tickets;    // zeroed counters: [tile][16 epilogue warps]
     int M, N, K, G;
-    int n_tiles;     // ceil(N / 128)
+    int n_tiles;     // NT = ceil(N / 128)
     int m_tiles;     // ceil(M / MT)
-    int split_k;     // >= 1
+    int split_k;     // 0: balanced chunks; S >= 1: classic Split-K
+    int nchunks;
     int stages;
 };
 
@@ -109,6 +127,18 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_ld4(uint32_t taddr, uint32_t (&r)[4]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(taddr)
+                 : "memory");
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -131,12 +161,64 @@ __host__ __device__ constexpr uint32_t tile_idesc(int mt) {
     return (1u << 4) | ((uint32_t)(mt >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
 }
 
-// K slice `sp` of `split_k` over G groups: first group and count (first G % split_k slices get one more).
-__device__ __forceinline__ void tile_slice(int G, int split_k, int sp, int& g0, int& ng) {
-    const int base = G / split_k, rem = G % split_k;
-    g0 = sp * base + min(sp, rem);
-    ng = base + (sp < rem ? 1 : 0);
+// ------------------------------------------------------------------ chunk schedule
+// First unit of chunk i (i == nchunks gives the end of the last chunk).
+__device__ __forceinline__ long long tile_chunk_begin(const TileParams& p, int i) {
+    if (p.split_k == 0) return ((long long)i * ((long long)p.m_tiles * p.n_tiles * p.G)) / p.nchunks;
+    const int t = i / p.split_k, s = i - t * p.split_k;
+    const int base = p.G / p.split_k, rem = p.G % p.split_k;
+    return (long long)t * p.G + s * base + min(s, rem);
 }
+// The chunk that holds unit u.
+__device__ __forceinline__ int tile_chunk_of(const TileParams& p, long long u) {
+    if (p.split_k == 0) return (int)(((u + 1) * p.nchunks - 1) / ((long long)p.m_tiles * p.n_tiles * p.G));
+    const int t = (int)(u / p.G), g = (int)(u - (long long)t * p.G);
+    const int base = p.G / p.split_k, rem = p.G % p.split_k;
+    const int s = (g < rem * (base + 1)) ? g / (base + 1) : rem + (g - rem * (base + 1)) / max(base, 1);
+    return t * p.split_k + s;
+}
+
+// Walks the 64-k stages of this CTA's chunks in order.  Every role of the CTA runs its own copy and
+// sees the same sequence.  Tile and group are kept incrementally (one division per chunk).
+struct StageWalk {
+    const TileParams& p;
+    int ci;                // current chunk
+    long long u0;          // first unit of the chunk
+    int t, g;              // current unit: tile (batch tile * NT + column tile) and group inside it
+    int t0, g0;            // the chunk's first unit
+    int left;              // units left in the chunk, the current one included
+    int c;                 // 64-k half of the unit's group
+    uint32_t n;            // stages walked so far (ring positions derive from it)
+    __device__ __forceinline__ StageWalk(const TileParams& p_)
+        : p(p_), ci((int)blockIdx.x), u0(0), t(0), g(0), t0(0), g0(0), left(0), c(0), n(0) {
+        load();
+    }
+    __device__ __forceinline__ void load() {
+        while (ci < p.nchunks) {
+            u0 = tile_chunk_begin(p, ci);
+            left = (int)(tile_chunk_begin(p, ci + 1) - u0);
+            if (left > 0) break;
+            ci += (int)gridDim.x;
+        }
+        t0 = t = (int)(u0 / p.G);
+        g0 = g = (int)(u0 - (long long)t * p.G);
+        c = 0;
+    }
+    __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
+    __device__ __forceinline__ void next() {
+        ++n;
+        if (c == 0) { c = 1; return; }
+        c = 0;
+        if (--left == 0) { ci += (int)gridDim.x; load(); return; }
+        if (++g == p.G) { g = 0; ++t; }
+    }
+    // first / last stage of a segment (the part of the chunk inside one tile)
+    __device__ __forceinline__ bool seg_first() const { return c == 0 && (g == 0 || (t == t0 && g == g0)); }
+    __device__ __forceinline__ bool seg_last() const { return c == 1 && (g == p.G - 1 || left == 1); }
+    // does the segment of the current stage start at the chunk's first unit / at the tile's first group
+    __device__ __forceinline__ bool seg_starts_chunk() const { return t == t0; }
+    __device__ __forceinline__ bool seg_starts_tile() const { return t != t0 || g0 == 0; }
+};
 
 template <int MT>
 __global__ void __launch_bounds__(kTileThreads, 1)
@@ -147,15 +229,18 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kStageBytes = tile_stage_bytes(MT);
     constexpr uint32_t kIdesc = tile_idesc(MT);
-    constexpr int kColsPerWarp = MT / 2;      // epilogue: two warps share a lane quarter
+    constexpr int kCW = MT / kTileSets;                  // accumulator columns (batch rows) per epilogue warp
+    constexpr int kDBufs = MT <= 128 ? 2 : 1;            // accumulators in TMEM
+    constexpr int kDStride = 128;                        // column distance between the two
+    constexpr uint32_t kWBytes = 2048u + 128u + 32u;     // per 64-column packed tile and stage
 
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [stages]  TMA landed
     uint64_t* empty = full + kTileMaxStages;                     // [stages]  MMAs that read the stage retired
     uint64_t* a_full = empty + kTileMaxStages;                   // [slots]   dequantized operand stored
     uint64_t* a_empty = a_full + kTileASlots;                    // [slots]   MMAs that read the slot retired
-    uint64_t* d_full = a_empty + kTileASlots;                    // accumulator complete
-    uint64_t* d_empty = d_full + 1;                              // accumulator drained by the epilogue
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(d_empty + 1);
+    uint64_t* d_full = a_empty + kTileASlots;                    // [2]       accumulator complete
+    uint64_t* d_empty = d_full + 2;                              // [2]       accumulator drained by the epilogue
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(d_empty + 2);
     int* flags = reinterpret_cast<int*>(tmem_slot + 1);          // [0] a bounded wait ran out, [1] stages issued
     unsigned char* stage0 = smem + kTileBarBytes;
 
@@ -171,8 +256,10 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             mbar_init(&a_full[i], 4);
             mbar_init(&a_empty[i], 1);
         }
-        mbar_init(d_full, 1);
-        mbar_init(d_empty, kTileDequantWarps);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&d_full[i], 1);
+            mbar_init(&d_empty[i], kTileDequantWarps);
+        }
         flags[0] = 0;
         flags[1] = 0;
         fence_mbar_init();
@@ -188,113 +275,130 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     volatile int* abort_flag = flags;
-
-    const int total_items = p.n_tiles * p.m_tiles * p.split_k;
+    // the next kernel in the stream may start its own prologue and weight prefetch
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
-            uint32_t n_stage = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
-                const int mt_i = item % p.m_tiles;
-                const int rest = item / p.m_tiles;
-                const int sp = rest % p.split_k;
-                const int nt = rest / p.split_k;
-                int g0, ng;
-                tile_slice(p.G, p.split_k, sp, g0, ng);
-                const int t0 = 2 * nt;                          // packed 64-column tiles t0, t0 + 1
-                const bool has_t1 = (t0 + 1) * kTileN < p.N;
-                const uint32_t tx = (has_t1 ? 2u : 1u) * (2048u + 128u + 32u) + (uint32_t)MT * 128u;
-                for (int st = 0; st < 2 * ng && ok; ++st, ++n_stage) {
-                    const int slot = n_stage % stages;
-                    const uint32_t ph = (n_stage / stages) & 1u;
+            auto issue_weights = [&](const StageWalk& w, unsigned char* sb, uint64_t* bar, int halves) {
+                const int nt = w.t % p.n_tiles;
+                const int g = w.g;
+                for (int h = 0; h < halves; ++h) {
+                    const size_t blk = (size_t)(2 * nt + h) * p.G + g;
+                    bulk_g2s(sb + kTileStageW + h * 2048, p.Wq + blk * kBlockWords + w.c * 512, 2048, bar);
+                    bulk_g2s(sb + kTileStageS + h * 128, p.S + blk * kSBlockHalves, 128, bar);
+                    bulk_g2s(sb + kTileStageZ + h * 32, p.Z + blk * kZBlockWords, 32, bar);
+                }
+            };
+            auto halves_of = [&](const StageWalk& w) {
+                const int nt = w.t % p.n_tiles;
+                return ((2 * nt + 1) * kTileN < p.N) ? 2 : 1;
+            };
+            auto issue_act = [&](const StageWalk& w, unsigned char* sb, uint64_t* bar) {
+                const int mt_i = w.t / p.n_tiles;
+                tma_load_2d(sb + kTileStageAct, &tmap_a, w.g * kGroup + w.c * kTileStageK, mt_i * MT, bar);
+            };
+            // 1. weights of the first ring-full of stages: they do not depend on the previous kernel
+            StageWalk pre(p);
+            while (pre.valid() && pre.n < (uint32_t)stages) {
+                unsigned char* sb = stage0 + (size_t)pre.n * kStageBytes;
+                const int halves = halves_of(pre);
+                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full[pre.n])),
+                             "r"(halves * kWBytes)
+                             : "memory");
+                issue_weights(pre, sb, &full[pre.n], halves);
+                pre.next();
+            }
+            // 2. everything else reads or writes memory the previous kernel may still be writing
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            StageWalk w(p);
+            for (; w.valid() && ok; w.next()) {
+                const int slot = w.n % stages;
+                unsigned char* sb = stage0 + (size_t)slot * kStageBytes;
+                if (w.n < (uint32_t)stages) {
+                    mbar_expect_tx(&full[slot], (uint32_t)MT * 128u);      // the arrival + the activation bytes
+                    issue_act(w, sb, &full[slot]);
+                } else {
+                    const uint32_t ph = (w.n / stages) & 1u;
                     if (!mbar_wait(&empty[slot], ph ^ 1u)) { ok = false; break; }
-                    const int g = g0 + (st >> 1), c = st & 1;
-                    unsigned char* sb = stage0 + (size_t)slot * kStageBytes;
-                    mbar_expect_tx(&full[slot], tx);
-                    for (int h = 0; h < (has_t1 ? 2 : 1); ++h) {
-                        const size_t blk = (size_t)(t0 + h) * p.G + g;
-                        bulk_g2s(sb + kTileStageW + h * 2048, p.Wq + blk * kBlockWords + c * 512, 2048, &full[slot]);
-                        bulk_g2s(sb + kTileStageS + h * 128, p.S + blk * kSBlockHalves, 128, &full[slot]);
-                        bulk_g2s(sb + kTileStageZ + h * 32, p.Z + blk * kZBlockWords, 32, &full[slot]);
-                    }
-                    tma_load_2d(sb + kTileStageAct, &tmap_a, g * kGroup + c * kTileStageK, mt_i * MT, &full[slot]);
+                    const int halves = halves_of(w);
+                    mbar_expect_tx(&full[slot], halves * kWBytes + (uint32_t)MT * 128u);
+                    issue_weights(w, sb, &full[slot], halves);
+                    issue_act(w, sb, &full[slot]);
                 }
             }
-            flags[1] = (int)n_stage;
+            flags[1] = (int)w.n;
             if (!ok) *abort_flag = 1;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (lane == 0) {
-            uint32_t n_stage = 0, n_item = 0;
+            uint32_t n_seg = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++n_item) {
-                const int sp = (item / p.m_tiles) % p.split_k;
-                int g0, ng;
-                tile_slice(p.G, p.split_k, sp, g0, ng);
-                // the epilogue of the previous item must have drained the accumulator
-                if (!mbar_wait(d_empty, (n_item & 1u) ^ 1u)) { ok = false; break; }
-                tc_fence_after();
-                for (int st = 0; st < 2 * ng; ++st, ++n_stage) {
-                    const int slot = n_stage % stages;
-                    const uint32_t ph = (n_stage / stages) & 1u;
-                    const int aslot = n_stage % kTileASlots;
-                    const uint32_t aph = (n_stage / kTileASlots) & 1u;
-                    if (!mbar_wait(&full[slot], ph) || !mbar_wait(&a_full[aslot], aph)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t act = smem_u32(stage0 + (size_t)slot * kStageBytes + kTileStageAct);
-                    const uint64_t bdesc = smem_desc_sw128(act);
-                    const uint32_t a_t = tmem_base + kTileAColBase + aslot * 32;
-#pragma unroll
-                    for (int kk = 0; kk < kTileStageK / 16; ++kk) {
-                        // 16 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled rows of B
-                        tc_mma_ts(tmem_base, a_t + kk * 8, bdesc + (uint64_t)(kk * 2), kIdesc, (st | kk) != 0 ? 1u : 0u);
-                    }
-                    tc_commit(&empty[slot]);
-                    tc_commit(&a_empty[aslot]);
+            for (StageWalk w(p); w.valid() && ok; w.next()) {
+                const int slot = w.n % stages;
+                const uint32_t ph = (w.n / stages) & 1u;
+                const int aslot = w.n % kTileASlots;
+                const uint32_t aph = (w.n / kTileASlots) & 1u;
+                const int dbuf = n_seg % kDBufs;
+                const bool first = w.seg_first();
+                if (first) {
+                    // the epilogue of the segment that used this accumulator before must have drained it
+                    if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
                 }
-                if (ok) tc_commit(d_full);
+                if (!mbar_wait(&full[slot], ph) || !mbar_wait(&a_full[aslot], aph)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t act = smem_u32(stage0 + (size_t)slot * kStageBytes + kTileStageAct);
+                const uint64_t bdesc = smem_desc_sw128(act);
+                const uint32_t a_t = tmem_base + kTileAColBase + aslot * 32;
+                const uint32_t d_t = tmem_base + dbuf * kDStride;
+#pragma unroll
+                for (int kk = 0; kk < kTileStageK / 16; ++kk) {
+                    // 16 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled rows of B
+                    tc_mma_ts(d_t, a_t + kk * 8, bdesc + (uint64_t)(kk * 2), kIdesc, (first && kk == 0) ? 0u : 1u);
+                }
+                tc_commit(&empty[slot]);
+                tc_commit(&a_empty[aslot]);
+                if (w.seg_last()) {
+                    tc_commit(&d_full[dbuf]);
+                    ++n_seg;
+                }
             }
             if (!ok) *abort_flag = 1;
         }
     } else {
         // ------------------------------------------------------------ dequant + epilogue warps
-        const int dw = warp - 2;               // 0..7
-        const int set = dw >> 2;               // stages with (index & 1) == set
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int dw = warp - 2;               // 0..15
+        const int set = dw >> 2;               // stages with (index % 4) == set
         const int quarter = warp & 3;          // TMEM lanes this warp may touch
         const int row = quarter * 32 + lane;   // column n inside the CTA tile = TMEM lane
         const int half = row >> 6, col = row & 63;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        // this thread's two 16-byte chunks of a 64-k line pair
-        const int woff0 = half * 2048 + (col >> 3) * 256 + (col & 7) * 16;
-        const int woff1 = half * 2048 + (col >> 3) * 256 + 128 + (((col & 7) + 4) & 7) * 16;
-        uint32_t n_stage = 0, n_item = 0;
+        // this thread's two 16-byte chunks of a 64-k line pair, its scale and its zero-point word
+        const int woff0 = kTileStageW + half * 2048 + (col >> 3) * 256 + (col & 7) * 16;
+        const int woff1 = kTileStageW + half * 2048 + (col >> 3) * 256 + 128 + (((col & 7) + 4) & 7) * 16;
+        const int soff = kTileStageS + row * 2;
+        const int zoff = kTileStageZ + (row >> 3) * 4;
+        const int zsh = 4 * (row & 7);
+        uint32_t n_seg = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++n_item) {
-            const int mt_i = item % p.m_tiles;
-            const int rest = item / p.m_tiles;
-            const int sp = rest % p.split_k;
-            const int nt = rest / p.split_k;
-            int g0, ng;
-            tile_slice(p.G, p.split_k, sp, g0, ng);
-            for (int st = 0; st < 2 * ng; ++st, ++n_stage) {
-                if ((int)(n_stage & 1u) != set) continue;
-                const int slot = n_stage % stages;
-                const uint32_t ph = (n_stage / stages) & 1u;
-                const int aslot = n_stage % kTileASlots;
-                const uint32_t aph = (n_stage / kTileASlots) & 1u;
-                if (!mbar_wait(&full[slot], ph) || !mbar_wait(&a_empty[aslot], aph ^ 1u)) { ok = false; break; }
-                tc_fence_after();
+        for (StageWalk w(p); w.valid() && ok; w.next()) {
+            if ((int)(w.n % kTileSets) == set) {
+                const int slot = w.n % stages;
+                const uint32_t ph = (w.n / stages) & 1u;
+                const int aslot = w.n % kTileASlots;
+                const uint32_t aph = (w.n / kTileASlots) & 1u;
+                if (!mbar_wait(&full[slot], ph)) { ok = false; break; }
                 const unsigned char* sb = stage0 + (size_t)slot * kStageBytes;
-                const uint4 w0 = *reinterpret_cast<const uint4*>(sb + kTileStageW + woff0);
-                const uint4 w1 = *reinterpret_cast<const uint4*>(sb + kTileStageW + woff1);
-                const __half s = *reinterpret_cast<const __half*>(sb + kTileStageS + row * 2);
-                const uint32_t zw = *reinterpret_cast<const uint32_t*>(sb + kTileStageZ + (row >> 3) * 4);
-                const uint32_t z = (zw >> (4 * (row & 7))) & 15u;
-                const __half2 s2 = __half2half2(s);
+                const uint4 w0 = *reinterpret_cast<const uint4*>(sb + woff0);
+                const uint4 w1 = *reinterpret_cast<const uint4*>(sb + woff1);
+                const __half2 s2 = __half2half2(*reinterpret_cast<const __half*>(sb + soff));
+                const uint32_t z = (*reinterpret_cast<const uint32_t*>(sb + zoff) >> zsh) & 15u;
                 const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
                 const uint32_t ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
                 uint32_t regs[32];
@@ -304,74 +408,83 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll
                     for (int j = 0; j < 4; ++j) regs[4 * i + j] = h2_as_u32(f.h[j]);
                 }
+                // the MMAs that read this operand slot eight stages ago must have retired
+                if (!mbar_wait(&a_empty[aslot], aph ^ 1u)) { ok = false; break; }
+                tc_fence_after();
                 tc_st32(tmem_base + lane_addr + kTileAColBase + aslot * 32, regs);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&a_full[aslot]);
             }
-            if (!ok) break;
+            if (!w.seg_last()) continue;
 
-            // ---------------------------------------------------- epilogue of this item
-            if (!mbar_wait(d_full, n_item & 1u)) { ok = false; break; }
+            // ---------------------------------------------------- epilogue of the segment that ends here
+            const int dbuf = n_seg % kDBufs;
+            if (!mbar_wait(&d_full[dbuf], (n_seg / kDBufs) & 1u)) { ok = false; break; }
+            ++n_seg;
             tc_fence_after();
+            const int T = w.t;
+            const int nt = T % p.n_tiles, mt_i = T / p.n_tiles;
             const int n = nt * kTileCols + row;
-            const int m_base = mt_i * MT;
-            const int col0 = set * kColsPerWarp;    // this warp's share of the accumulator columns
-            if (p.split_k == 1) {
+            const int m_base = mt_i * MT + set * kCW;     // first batch row of this warp's columns
+            const uint32_t d_t = tmem_base + lane_addr + dbuf * kDStride + set * kCW;
+            const long long tile_u0 = (long long)T * p.G;
+            const bool whole = w.seg_starts_tile() && (w.g == p.G - 1);
+            // first segment of a chunk -> slot 2 ci, its continuation into a later tile -> 2 ci + 1
+            float* part = p.ws + ((size_t)(2 * w.ci + (w.seg_starts_chunk() ? 0 : 1)) * MT + set * kCW) * kTileCols + row;
+            constexpr int kStep = kCW >= 16 ? 16 : kCW;
 #pragma unroll 1
-                for (int cc = 0; cc < kColsPerWarp; cc += 16) {
-                    uint32_t v[16];
-                    tc_ld16(tmem_base + lane_addr + col0 + cc, v);
-                    tc_wait_ld();
+            for (int cc = 0; cc < kCW; cc += kStep) {
+                uint32_t v[kStep];
+                if constexpr (kStep == 16) tc_ld16(d_t + cc, v);
+                else if constexpr (kStep == 8) tc_ld8(d_t + cc, v);
+                else tc_ld4(d_t + cc, v);
+                tc_wait_ld();
+                if (whole) {
                     if (n < p.N) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int m = m_base + col0 + cc + j;
+                        for (int j = 0; j < kStep; ++j) {
+                            const int m = m_base + cc + j;
                             if (m < p.M) p.C[(size_t)m * p.N + n] = __float2half_rn(__uint_as_float(v[j]));
                         }
                     }
-                }
-            } else {
-                float* slot_ws = p.ws + (size_t)item * (MT * kTileCols);
-#pragma unroll 1
-                for (int cc = 0; cc < kColsPerWarp; cc += 16) {
-                    uint32_t v[16];
-                    tc_ld16(tmem_base + lane_addr + col0 + cc, v);
-                    tc_wait_ld();
+                } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        slot_ws[(size_t)(col0 + cc + j) * kTileCols + row] = __uint_as_float(v[j]);
+                    for (int j = 0; j < kStep; ++j) part[(size_t)(cc + j) * kTileCols] = __uint_as_float(v[j]);
                 }
             }
-            // accumulator drained: the next item's first MMA may overwrite it
+            // accumulator drained: a later segment's first MMA may overwrite it
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(d_empty);
+            if (lane == 0) mbar_arrive(&d_empty[dbuf]);
 
-            if (p.split_k > 1) {
-                // Split-K reduce (Algorithm 1, Phase 3), per warp region (32 columns n x MT/2 rows m): the
-                // warp that draws the region's last ticket adds the S partial regions in ascending slice
-                // order and casts to FP16.  No warp waits for another CTA.
+            if (!whole) {
+                // Split-K reduce (Algorithm 1, Phase 3), per warp region (32 columns n x MT/4 rows m)
                 __threadfence();
                 __syncwarp();
-                int* ticket = p.tickets + ((size_t)(nt * p.m_tiles + mt_i) * kTileDequantWarps + dw);
+                const int c_first = tile_chunk_of(p, tile_u0);
+                const int c_last = tile_chunk_of(p, tile_u0 + p.G - 1);
+                int* ticket = p.tickets + ((size_t)T * kTileDequantWarps + dw);
                 int last = 0;
                 if (lane == 0) {
                     const int old = atomicAdd(ticket, 1);
-                    last = (old == p.split_k - 1);
+                    last = (old == c_last - c_first);
                     if (last) *ticket = 0;   // every contributor has arrived: zero for the next call
                 }
                 last = __shfl_sync(0xffffffffu, last, 0);
                 if (last) {
                     __threadfence();
-                    // items of this tile: ((nt * split_k + s) * m_tiles + mt_i), s = 0 .. split_k - 1
-                    const float* base = p.ws + ((size_t)nt * p.split_k * p.m_tiles + mt_i) * (MT * kTileCols) + row;
-                    const size_t s_stride = (size_t)p.m_tiles * (MT * kTileCols);
-#pragma unroll 4
-                    for (int mm = col0; mm < col0 + kColsPerWarp; ++mm) {
-                        float acc = 0.f;
-                        for (int s = 0; s < p.split_k; ++s) acc += __ldcg(base + s * s_stride + (size_t)mm * kTileCols);
+                    // contributors in ascending K: chunk c_first (its first segment if it starts at the tile's
+                    // first unit, else its continuation), then the first segments of the others
+                    const size_t slot_elems = (size_t)MT * kTileCols;
+                    const float* base = p.ws + (size_t)(set * kCW) * kTileCols + row;
+                    const size_t first_slot = 2 * (size_t)c_first + (tile_chunk_begin(p, c_first) == tile_u0 ? 0 : 1);
+#pragma unroll 2
+                    for (int mm = 0; mm < kCW; ++mm) {
+                        float acc = __ldcg(base + first_slot * slot_elems + (size_t)mm * kTileCols);
+                        for (int c = c_first + 1; c <= c_last; ++c)
+                            acc += __ldcg(base + (size_t)(2 * c) * slot_elems + (size_t)mm * kTileCols);
                         const int m = m_base + mm;
                         if (m < p.M && n < p.N) p.C[(size_t)m * p.N + n] = __float2half_rn(acc);
                     }

@@ -114,8 +114,8 @@ def test_workspace_errors():
     with pytest.raises(B.W4A16Error) as e:
         B.w4a16_gemm(A, pw, split_k=4, path=B.PATH_DECODE)
     assert e.value.code == -5
-    small = torch.empty(32768, dtype=torch.uint8, device="cuda")
-    B.w4a16_set_workspace(small[(-small.data_ptr()) % 256:][:16384 + 256])
+    small = torch.empty(B.WS_HEADER_BYTES + 1024, dtype=torch.uint8, device="cuda")
+    B.w4a16_set_workspace(small[(-small.data_ptr()) % 256:][:B.WS_HEADER_BYTES + 256])
     with pytest.raises(B.W4A16Error) as e:
         B.w4a16_gemm(A, pw, split_k=4, path=B.PATH_DECODE)
     assert e.value.code == -5

@@ -23,9 +23,9 @@ def _run(d, M, N, K, split_k, path=B.PATH_TILE):
     return C
 
 
-# (M, K, N): batch tiles of 32 / 64 / 128 / 256 rows with ragged tails, one and several column
+# (M, K, N): batch tiles of 16 / 32 / 64 / 128 / 256 rows with ragged tails, one and several column
 # tiles, a 64-column tail tile (N = 192, 320), one to many groups
-SHAPES = [(32, 128, 128), (1, 256, 128), (17, 640, 192), (33, 384, 256), (64, 1152, 128),
+SHAPES = [(32, 128, 128), (1, 256, 128), (9, 640, 192), (16, 1152, 256), (17, 640, 192), (33, 384, 256), (64, 1152, 128),
           (100, 896, 320), (128, 512, 256), (129, 768, 128), (256, 2048, 384), (300, 1280, 192),
           (700, 640, 256)]
 
@@ -41,13 +41,16 @@ def test_tile_path_matches_oracle(M, K, N, split_k):
     assert_close(c_f64(C), ref, "tile M%d K%d N%d S%d" % (M, K, N, split_k))
 
 
-def test_tile_path_many_items_per_cta():
-    # more (tile, slice) items than SMs: every CTA walks several items through the same rings
+@pytest.mark.parametrize("split_k", [2, 0, 1])
+def test_tile_path_many_chunks_per_cta(split_k):
+    # more tiles than SMs.  Classic split: every CTA walks several chunks through the same rings.
+    # Balanced: a chunk is about 2.2 units of a 2-unit tile, so chunks hold whole tiles and partial
+    # segments of both neighbours.
     M, K, N = 40, 256, 128 * 160
     d = wl.make_problem(M, K, N, seed=7100)
-    C = _run(d, M, N, K, 2)
+    C = _run(d, M, N, K, split_k)
     ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
-    assert_close(c_f64(C), ref, "tile many items")
+    assert_close(c_f64(C), ref, "tile many chunks, split_k=%d" % split_k)
 
 
 def test_tile_path_exact_inputs_bit_equal_for_every_split():
