@@ -73,26 +73,39 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait: returns false (after recording the status code) if the phase never completes.
+// The whole poll loop is one asm block (a predicate branch straight off try_wait; about 40 clocks
+// when the phase is already complete).  try_wait itself blocks for a hardware-defined slice, so
+// the limit below is far beyond any legitimate wait, yet finite.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .u32 cnt;\n\t"
+        "mov.u32 cnt, 0;\n\t"
+        "W4A16_WAIT_LOOP:\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
+        "@p bra W4A16_WAIT_DONE;\n\t"
+        "add.u32 cnt, cnt, 1;\n\t"
+        "setp.lt.u32 q, cnt, 0x400000;\n\t"
+        "@q bra W4A16_WAIT_LOOP;\n\t"
+        "W4A16_WAIT_DONE:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
+    if (ok == 0) report_status(kStatusMbarTimeout);
     return ok != 0;
 }
-// Bounded wait: returns false (after recording the status code) if the phase never
-// completes.  try_wait itself blocks for a hardware-defined slice, so the limit below is
-// far beyond any legitimate wait (seconds), yet finite.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-    }
-    report_status(kStatusMbarTimeout);
-    return false;
+
+// One lane of a converged warp (warp-uniform control flow keeps addresses and descriptors in
+// uniform registers; only the issuing instruction itself is predicated on the elected lane).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 // TMA bulk copy global -> shared (1-D, no tensor map).  Addresses and size are multiples

@@ -3,15 +3,16 @@
 // The product is computed transposed, C^T[n, m] = sum_k W16[k, n] A[m, k], so that the
 // DEQUANTIZED WEIGHTS are the MMA's 128-row A operand and live only in tensor memory:
 //
-//   HBM --TMA bulk--> shared (packed nibbles, scales, zeros)          producer warp
-//   shared -> registers: unpack, (q - z) exact, * s in FP16            8 dequant warps
+//   HBM --128-bit loads--> registers (packed nibbles, scale, zero)    16 dequant warps,
+//   registers: unpack, (q - z) exact, * s in FP16                      one column n per thread
 //   registers --tcgen05.st--> TMEM (A operand, one column n per lane, k packed along columns)
 //   HBM --TMA tensor (128B swizzle)--> shared (activation tile, MT rows m x 64 k): B operand
-//   tcgen05.mma.kind::f16  D[128 n x MT m] (FP32, TMEM) += A(TMEM) . B(shared)   one thread
+//   tcgen05.mma.kind::f16  D[128 n x MT m] (FP32, TMEM) += A(TMEM) . B(shared)   one elected lane
 //   TMEM --tcgen05.ld--> registers -> FP16 C, or FP32 partial tile + ticket (Split-K)
 //
-// so dequantized weights never touch shared or global memory (Algorithm 1's Phase 1 output
-// stays on chip), and the activation tile is re-used by all 128 columns of the CTA tile.
+// so packed weights go from HBM straight to registers, dequantized weights never touch shared or
+// global memory (Algorithm 1's Phase 1 output stays on chip), and the activation tile is re-used
+// by all 128 columns of the CTA tile.
 //
 // Work is counted in units: one unit = 128 columns x one group (128 k) of one batch tile, numbered
 // U = (batch tile * NT + column tile) * G + group.  The unit range is cut into chunks, each CTA of
@@ -27,14 +28,17 @@
 // No warp ever waits for another CTA, and the order of the sum is fixed, so results are
 // bit-identical from run to run.
 //
-// One pipeline stage is 64 k: 4 KiB of nibbles, the group's scales and zeros, and an MT x 64 FP16
-// activation box.  Four sets of four dequant warps take stages round-robin; inside a set warp w
-// owns TMEM lanes 32 (w % 4) .. + 31, one column n per thread.  With MT <= 128 two accumulators
-// alternate between segments, so one drains while the next fills.  The packed weights do not
-// depend on the previous kernel in the stream: under programmatic dependent launch the producer
-// fills the whole ring with them before griddepcontrol.wait, and only activations, C and the
-// workspace are touched after it.  All waits are bounded mbarrier waits; a wait that runs out
-// records a status code and the CTA drains and exits (TMEM is always released).
+// One pipeline stage is 64 k.  A ring of R <= 8 slots holds, per slot, the MT x 64 FP16 activation
+// box in shared memory and 32 TMEM columns of dequantized weights; the MMAs of a stage release both
+// with one commit.  Four sets of four dequant warps take stages round-robin; inside a set warp w
+// owns TMEM lanes 32 (w % 4) .. + 31.  Each thread keeps the packed words of its next few stages in
+// registers (loads issued that far ahead).  With MT <= 128 two accumulators alternate between
+// segments, so one drains while the next fills.  The packed weights do not depend on the previous
+// kernel in the stream: under programmatic dependent launch the first weight loads are issued
+// before griddepcontrol.wait, and only activations, C and the workspace are touched after it.
+// The producer and MMA warps run warp-uniform loops and elect one lane per instruction, which
+// keeps descriptors in uniform registers.  All waits are bounded mbarrier waits; a wait that runs
+// out records a status code and the CTA drains and exits (TMEM is always released).
 #pragma once
 
 #include <cuda.h>
@@ -48,16 +52,12 @@ constexpr int kTileStageK = 64;                     // k per pipeline stage
 constexpr int kTileDequantWarps = 16;               // four sets of four (one warp per TMEM lane quarter)
 constexpr int kTileSets = kTileDequantWarps / 4;
 constexpr int kTileThreads = (2 + kTileDequantWarps) * 32;   // producer, MMA, dequant/epilogue warps
-constexpr int kTileASlots = 8;                      // TMEM ring of A-operand slots (32 columns each)
+constexpr int kTileMaxStages = 8;                   // ring slots: activation box + 32 TMEM columns each
 constexpr int kTileAColBase = 256;                  // accumulators in columns [0, 256), the ring in [256, 512)
-constexpr int kTileStageW = 0;                      // 2 x 2 KiB of nibbles (two 64-column packed tiles)
-constexpr int kTileStageS = 4096;                   // 2 x 64 FP16
-constexpr int kTileStageZ = 4352;                   // 2 x 8 uint32
-constexpr int kTileStageAct = 5120;                 // MT x 128 B, 1024-byte aligned (128B swizzle atom)
-constexpr int kTileMaxStages = 16;
+constexpr int kTilePrefetch = 3;                    // stages of packed words a dequant thread holds in registers
 constexpr int kTileBarBytes = 1024;
 
-__host__ __device__ constexpr int tile_stage_bytes(int mt) { return kTileStageAct + mt * 128; }
+__host__ __device__ constexpr int tile_stage_bytes(int mt) { return mt * 128; }
 
 struct TileParams {
     const uint32_t* Wq;
@@ -106,6 +106,13 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
         "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
         "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -179,21 +186,29 @@ __device__ __forceinline__ int tile_chunk_of(const TileParams& p, long long u) {
 }
 
 // Walks the 64-k stages of this CTA's chunks in order.  Every role of the CTA runs its own copy and
-// sees the same sequence.  Tile and group are kept incrementally (one division per chunk).
+// sees the same sequence.  The single-thread roles (TMA producer, MMA issuer) sit on the critical
+// path of every stage, so everything here is kept incrementally: no division or 64-bit arithmetic
+// per stage, only once per chunk.
 struct StageWalk {
     const TileParams& p;
     int ci;                // current chunk
-    long long u0;          // first unit of the chunk
     int t, g;              // current unit: tile (batch tile * NT + column tile) and group inside it
+    int nt, mt_i;          // t % NT, t / NT
     int t0, g0;            // the chunk's first unit
     int left;              // units left in the chunk, the current one included
     int c;                 // 64-k half of the unit's group
-    uint32_t n;            // stages walked so far (ring positions derive from it)
+    bool first_unit;       // still on the chunk's first unit
+    uint32_t n;            // stages walked so far
+    int slot;              // n % stages
+    uint32_t ph;           // (n / stages) & 1
+    const int stages;
     __device__ __forceinline__ StageWalk(const TileParams& p_)
-        : p(p_), ci((int)blockIdx.x), u0(0), t(0), g(0), t0(0), g0(0), left(0), c(0), n(0) {
+        : p(p_), ci((int)blockIdx.x), t(0), g(0), nt(0), mt_i(0), t0(0), g0(0), left(0), c(0), first_unit(true),
+          n(0), slot(0), ph(0), stages(p_.stages) {
         load();
     }
     __device__ __forceinline__ void load() {
+        long long u0 = 0;
         while (ci < p.nchunks) {
             u0 = tile_chunk_begin(p, ci);
             left = (int)(tile_chunk_begin(p, ci + 1) - u0);
@@ -202,22 +217,38 @@ struct StageWalk {
         }
         t0 = t = (int)(u0 / p.G);
         g0 = g = (int)(u0 - (long long)t * p.G);
+        mt_i = t / p.n_tiles;
+        nt = t - mt_i * p.n_tiles;
         c = 0;
+        first_unit = true;
     }
     __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
     __device__ __forceinline__ void next() {
         ++n;
+        if (++slot == stages) { slot = 0; ph ^= 1u; }
         if (c == 0) { c = 1; return; }
         c = 0;
         if (--left == 0) { ci += (int)gridDim.x; load(); return; }
-        if (++g == p.G) { g = 0; ++t; }
+        first_unit = false;
+        if (++g == p.G) {
+            g = 0;
+            ++t;
+            if (++nt == p.n_tiles) { nt = 0; ++mt_i; }
+        }
     }
     // first / last stage of a segment (the part of the chunk inside one tile)
-    __device__ __forceinline__ bool seg_first() const { return c == 0 && (g == 0 || (t == t0 && g == g0)); }
+    __device__ __forceinline__ bool seg_first() const { return c == 0 && (g == 0 || first_unit); }
     __device__ __forceinline__ bool seg_last() const { return c == 1 && (g == p.G - 1 || left == 1); }
     // does the segment of the current stage start at the chunk's first unit / at the tile's first group
     __device__ __forceinline__ bool seg_starts_chunk() const { return t == t0; }
     __device__ __forceinline__ bool seg_starts_tile() const { return t != t0 || g0 == 0; }
+};
+
+// Packed words, scale and zero point of one thread's column for one 64-k stage.
+struct StageRegs {
+    uint4 w0, w1;     // k = 0..31 and 32..63 of the stage
+    uint32_t s;       // FP16 scale bits
+    uint32_t zw;      // zero-point word of the column's 8-column block
 };
 
 template <int MT>
@@ -232,14 +263,12 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     constexpr int kCW = MT / kTileSets;                  // accumulator columns (batch rows) per epilogue warp
     constexpr int kDBufs = MT <= 128 ? 2 : 1;            // accumulators in TMEM
     constexpr int kDStride = 128;                        // column distance between the two
-    constexpr uint32_t kWBytes = 2048u + 128u + 32u;     // per 64-column packed tile and stage
 
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [stages]  TMA landed
-    uint64_t* empty = full + kTileMaxStages;                     // [stages]  MMAs that read the stage retired
-    uint64_t* a_full = empty + kTileMaxStages;                   // [slots]   dequantized operand stored
-    uint64_t* a_empty = a_full + kTileASlots;                    // [slots]   MMAs that read the slot retired
-    uint64_t* d_full = a_empty + kTileASlots;                    // [2]       accumulator complete
-    uint64_t* d_empty = d_full + 2;                              // [2]       accumulator drained by the epilogue
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [R]  activation box landed
+    uint64_t* a_full = full + kTileMaxStages;                    // [R]  dequantized operand stored in TMEM
+    uint64_t* retired = a_full + kTileMaxStages;                 // [R]  the stage's MMAs retired: slot free
+    uint64_t* d_full = retired + kTileMaxStages;                 // [2]  accumulator complete
+    uint64_t* d_empty = d_full + 2;                              // [2]  accumulator drained by the epilogue
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(d_empty + 2);
     int* flags = reinterpret_cast<int*>(tmem_slot + 1);          // [0] a bounded wait ran out, [1] stages issued
     unsigned char* stage0 = smem + kTileBarBytes;
@@ -250,11 +279,8 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
             mbar_init(&full[i], 1);
-            mbar_init(&empty[i], 1);
-        }
-        for (int i = 0; i < kTileASlots; ++i) {
             mbar_init(&a_full[i], 4);
-            mbar_init(&a_empty[i], 1);
+            mbar_init(&retired[i], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&d_full[i], 1);
@@ -279,143 +305,152 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
-        // ------------------------------------------------------------ producer
+        // ------------------------------------------------------------ producer: activation boxes
+        if (elect_one()) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // activations may come from the previous kernel
+        bool ok = true;
+        StageWalk w(p);
+        for (; w.valid(); w.next()) {
+            const int slot = w.slot;
+            if (w.n >= (uint32_t)stages && !mbar_wait(&retired[slot], w.ph ^ 1u)) { ok = false; break; }
+            if (elect_one()) {
+                mbar_expect_tx(&full[slot], (uint32_t)MT * 128u);
+                tma_load_2d(stage0 + (size_t)slot * kStageBytes, &tmap_a, w.g * kGroup + w.c * kTileStageK, w.mt_i * MT,
+                            &full[slot]);
+            }
+            __syncwarp();
+        }
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
-            bool ok = true;
-            auto issue_weights = [&](const StageWalk& w, unsigned char* sb, uint64_t* bar, int halves) {
-                const int nt = w.t % p.n_tiles;
-                const int g = w.g;
-                for (int h = 0; h < halves; ++h) {
-                    const size_t blk = (size_t)(2 * nt + h) * p.G + g;
-                    bulk_g2s(sb + kTileStageW + h * 2048, p.Wq + blk * kBlockWords + w.c * 512, 2048, bar);
-                    bulk_g2s(sb + kTileStageS + h * 128, p.S + blk * kSBlockHalves, 128, bar);
-                    bulk_g2s(sb + kTileStageZ + h * 32, p.Z + blk * kZBlockWords, 32, bar);
-                }
-            };
-            auto halves_of = [&](const StageWalk& w) {
-                const int nt = w.t % p.n_tiles;
-                return ((2 * nt + 1) * kTileN < p.N) ? 2 : 1;
-            };
-            auto issue_act = [&](const StageWalk& w, unsigned char* sb, uint64_t* bar) {
-                const int mt_i = w.t / p.n_tiles;
-                tma_load_2d(sb + kTileStageAct, &tmap_a, w.g * kGroup + w.c * kTileStageK, mt_i * MT, bar);
-            };
-            // 1. weights of the first ring-full of stages: they do not depend on the previous kernel
-            StageWalk pre(p);
-            while (pre.valid() && pre.n < (uint32_t)stages) {
-                unsigned char* sb = stage0 + (size_t)pre.n * kStageBytes;
-                const int halves = halves_of(pre);
-                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full[pre.n])),
-                             "r"(halves * kWBytes)
-                             : "memory");
-                issue_weights(pre, sb, &full[pre.n], halves);
-                pre.next();
-            }
-            // 2. everything else reads or writes memory the previous kernel may still be writing
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            StageWalk w(p);
-            for (; w.valid() && ok; w.next()) {
-                const int slot = w.n % stages;
-                unsigned char* sb = stage0 + (size_t)slot * kStageBytes;
-                if (w.n < (uint32_t)stages) {
-                    mbar_expect_tx(&full[slot], (uint32_t)MT * 128u);      // the arrival + the activation bytes
-                    issue_act(w, sb, &full[slot]);
-                } else {
-                    const uint32_t ph = (w.n / stages) & 1u;
-                    if (!mbar_wait(&empty[slot], ph ^ 1u)) { ok = false; break; }
-                    const int halves = halves_of(w);
-                    mbar_expect_tx(&full[slot], halves * kWBytes + (uint32_t)MT * 128u);
-                    issue_weights(w, sb, &full[slot], halves);
-                    issue_act(w, sb, &full[slot]);
-                }
-            }
             flags[1] = (int)w.n;
             if (!ok) *abort_flag = 1;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (lane == 0) {
-            uint32_t n_seg = 0;
-            bool ok = true;
-            for (StageWalk w(p); w.valid() && ok; w.next()) {
-                const int slot = w.n % stages;
-                const uint32_t ph = (w.n / stages) & 1u;
-                const int aslot = w.n % kTileASlots;
-                const uint32_t aph = (w.n / kTileASlots) & 1u;
-                const int dbuf = n_seg % kDBufs;
-                const bool first = w.seg_first();
-                if (first) {
-                    // the epilogue of the segment that used this accumulator before must have drained it
-                    if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
-                }
-                if (!mbar_wait(&full[slot], ph) || !mbar_wait(&a_full[aslot], aph)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t act = smem_u32(stage0 + (size_t)slot * kStageBytes + kTileStageAct);
-                const uint64_t bdesc = smem_desc_sw128(act);
-                const uint32_t a_t = tmem_base + kTileAColBase + aslot * 32;
+        uint32_t n_seg = 0;
+        bool ok = true;
+        for (StageWalk w(p); w.valid(); w.next()) {
+            const int slot = w.slot;
+            const int dbuf = n_seg % kDBufs;
+            const bool first = w.seg_first();
+            if (first) {
+                // the epilogue of the segment that used this accumulator before must have drained it
+                if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
+            }
+            if (!mbar_wait(&full[slot], w.ph) || !mbar_wait(&a_full[slot], w.ph)) { ok = false; break; }
+            tc_fence_after();
+            const bool last = w.seg_last();
+            if (elect_one()) {
+                const uint64_t bdesc = smem_desc_sw128(smem_u32(stage0 + (size_t)slot * kStageBytes));
+                const uint32_t a_t = tmem_base + kTileAColBase + slot * 32;
                 const uint32_t d_t = tmem_base + dbuf * kDStride;
 #pragma unroll
                 for (int kk = 0; kk < kTileStageK / 16; ++kk) {
                     // 16 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled rows of B
                     tc_mma_ts(d_t, a_t + kk * 8, bdesc + (uint64_t)(kk * 2), kIdesc, (first && kk == 0) ? 0u : 1u);
                 }
-                tc_commit(&empty[slot]);
-                tc_commit(&a_empty[aslot]);
-                if (w.seg_last()) {
-                    tc_commit(&d_full[dbuf]);
-                    ++n_seg;
-                }
+                tc_commit(&retired[slot]);
+                if (last) tc_commit(&d_full[dbuf]);
             }
-            if (!ok) *abort_flag = 1;
+            __syncwarp();
+            if (last) ++n_seg;
         }
+        if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------ dequant + epilogue warps
-        asm volatile("griddepcontrol.wait;" ::: "memory");
         const int dw = warp - 2;               // 0..15
         const int set = dw >> 2;               // stages with (index % 4) == set
         const int quarter = warp & 3;          // TMEM lanes this warp may touch
         const int row = quarter * 32 + lane;   // column n inside the CTA tile = TMEM lane
         const int half = row >> 6, col = row & 63;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        // this thread's two 16-byte chunks of a 64-k line pair, its scale and its zero-point word
-        const int woff0 = kTileStageW + half * 2048 + (col >> 3) * 256 + (col & 7) * 16;
-        const int woff1 = kTileStageW + half * 2048 + (col >> 3) * 256 + 128 + (((col & 7) + 4) & 7) * 16;
-        const int soff = kTileStageS + row * 2;
-        const int zoff = kTileStageZ + (row >> 3) * 4;
-        const int zsh = 4 * (row & 7);
+        // word offsets of this thread's two 16-byte chunks inside a block's 64-k half
+        const int wo0 = (col >> 3) * 64 + (col & 7) * 4;
+        const int wo1 = (col >> 3) * 64 + 32 + (((col & 7) + 4) & 7) * 4;
+        const int zsh = 4 * (col & 7);
+
+        // packed words of the stage the load walker stands on (zeros past the matrix edge)
+        auto load_stage = [&](const StageWalk& w, StageRegs& r) {
+            const int t64 = 2 * w.nt + half;                      // 64-column packed tile
+            if (t64 * kTileN < p.N) {
+                const size_t blk = (size_t)t64 * p.G + w.g;
+                const uint32_t* wp = p.Wq + blk * kBlockWords + w.c * 512;
+                r.w0 = __ldg(reinterpret_cast<const uint4*>(wp + wo0));
+                r.w1 = __ldg(reinterpret_cast<const uint4*>(wp + wo1));
+                r.s = __ldg(reinterpret_cast<const unsigned short*>(p.S) + blk * kSBlockHalves + col);
+                r.zw = __ldg(p.Z + blk * kZBlockWords + (col >> 3));
+            } else {
+                r.w0 = make_uint4(0, 0, 0, 0);
+                r.w1 = make_uint4(0, 0, 0, 0);
+                r.s = 0;
+                r.zw = 0;
+            }
+        };
+        // advance a walker to this set's next stage at or after its position
+        auto seek_own = [&](StageWalk& w) {
+            while (w.valid() && (int)(w.n % kTileSets) != set) w.next();
+        };
+
+        StageRegs pf[kTilePrefetch];
+        StageWalk wl(p);
+        seek_own(wl);
+#pragma unroll
+        for (int i = 0; i < kTilePrefetch; ++i) {
+            if (wl.valid()) {
+                load_stage(wl, pf[i]);
+                wl.next();
+                seek_own(wl);
+            }
+        }
+        // everything below may read or write memory the previous kernel is still writing
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+
         uint32_t n_seg = 0;
         bool ok = true;
         for (StageWalk w(p); w.valid() && ok; w.next()) {
             if ((int)(w.n % kTileSets) == set) {
-                const int slot = w.n % stages;
-                const uint32_t ph = (w.n / stages) & 1u;
-                const int aslot = w.n % kTileASlots;
-                const uint32_t aph = (w.n / kTileASlots) & 1u;
-                if (!mbar_wait(&full[slot], ph)) { ok = false; break; }
-                const unsigned char* sb = stage0 + (size_t)slot * kStageBytes;
-                const uint4 w0 = *reinterpret_cast<const uint4*>(sb + woff0);
-                const uint4 w1 = *reinterpret_cast<const uint4*>(sb + woff1);
-                const __half2 s2 = __half2half2(*reinterpret_cast<const __half*>(sb + soff));
-                const uint32_t z = (*reinterpret_cast<const uint32_t*>(sb + zoff) >> zsh) & 15u;
-                const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
-                const uint32_t ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-                uint32_t regs[32];
+                const int slot = w.slot;
+                const StageRegs cur = pf[0];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) regs[4 * i + j] = h2_as_u32(f.h[j]);
+                for (int i = 0; i + 1 < kTilePrefetch; ++i) pf[i] = pf[i + 1];
+                if (wl.valid()) {
+                    load_stage(wl, pf[kTilePrefetch - 1]);
+                    wl.next();
+                    seek_own(wl);
                 }
-                // the MMAs that read this operand slot eight stages ago must have retired
-                if (!mbar_wait(&a_empty[aslot], aph ^ 1u)) { ok = false; break; }
+                const uint32_t z = (cur.zw >> zsh) & 15u;
+                const __half2 s2 = u32_as_h2(cur.s * 0x00010001u);
+                const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
+                // the MMAs that read this slot one ring turn ago must have retired
+                if (w.n >= (uint32_t)stages && !mbar_wait(&retired[slot], w.ph ^ 1u)) { ok = false; break; }
                 tc_fence_after();
-                tc_st32(tmem_base + lane_addr + kTileAColBase + aslot * 32, regs);
+                const uint32_t a_t = tmem_base + lane_addr + kTileAColBase + slot * 32;
+                {
+                    const uint32_t ww[4] = {cur.w0.x, cur.w0.y, cur.w0.z, cur.w0.w};   // k = 0 .. 31
+                    uint32_t regs[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) regs[4 * i + j] = h2_as_u32(f.h[j]);
+                    }
+                    tc_st16(a_t, regs);
+                }
+                {
+                    const uint32_t ww[4] = {cur.w1.x, cur.w1.y, cur.w1.z, cur.w1.w};   // k = 32 .. 63
+                    uint32_t regs[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) regs[4 * i + j] = h2_as_u32(f.h[j]);
+                    }
+                    tc_st16(a_t + 16, regs);
+                }
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[aslot]);
+                if (lane == 0) mbar_arrive(&a_full[slot]);
             }
             if (!w.seg_last()) continue;
 
@@ -425,7 +460,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             ++n_seg;
             tc_fence_after();
             const int T = w.t;
-            const int nt = T % p.n_tiles, mt_i = T / p.n_tiles;
+            const int nt = w.nt, mt_i = w.mt_i;
             const int n = nt * kTileCols + row;
             const int m_base = mt_i * MT + set * kCW;     // first batch row of this warp's columns
             const uint32_t d_t = tmem_base + lane_addr + dbuf * kDStride + set * kCW;
@@ -491,7 +526,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 }
             }
         }
-        if (!ok) *abort_flag = 1;
+        if (!ok && lane == 0) *abort_flag = 1;
     }
 
     // ---------------------------------------------------------------- teardown
