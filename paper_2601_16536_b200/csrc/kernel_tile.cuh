@@ -185,63 +185,70 @@ __device__ __forceinline__ int tile_chunk_of(const TileParams& p, long long u) {
     return t * p.split_k + s;
 }
 
-// Walks the 64-k stages of this CTA's chunks in order.  Every role of the CTA runs its own copy and
-// sees the same sequence.  The single-thread roles (TMA producer, MMA issuer) sit on the critical
-// path of every stage, so everything here is kept incrementally: no division or 64-bit arithmetic
-// per stage, only once per chunk.
-struct StageWalk {
+// Walks the segments of this CTA's chunks in order (a segment = the part of a chunk inside one
+// tile).  Every role of the CTA runs its own copy and sees the same sequence.  A warp runs dependent
+// scalar code at only one instruction every several clocks, and the producer and MMA warps sit on
+// the critical path of every stage: so all per-stage work of the roles is a plain counted loop over
+// the segment's 2 * units stages, and the divisions and 64-bit arithmetic happen here, once per chunk.
+struct SegWalk {
     const TileParams& p;
-    int ci;                // current chunk
-    int t, g;              // current unit: tile (batch tile * NT + column tile) and group inside it
-    int nt, mt_i;          // t % NT, t / NT
-    int t0, g0;            // the chunk's first unit
-    int left;              // units left in the chunk, the current one included
-    int c;                 // 64-k half of the unit's group
-    bool first_unit;       // still on the chunk's first unit
-    uint32_t n;            // stages walked so far
-    int slot;              // n % stages
-    uint32_t ph;           // (n / stages) & 1
-    const int stages;
-    __device__ __forceinline__ StageWalk(const TileParams& p_)
-        : p(p_), ci((int)blockIdx.x), t(0), g(0), nt(0), mt_i(0), t0(0), g0(0), left(0), c(0), first_unit(true),
-          n(0), slot(0), ph(0), stages(p_.stages) {
-        load();
+    int ci;            // current chunk
+    int t;             // tile = batch tile * NT + column tile
+    int nt, mt_i;      // t % NT, t / NT
+    int g0;            // first group of the segment inside the tile
+    int units;         // groups in the segment
+    int left;          // units of the chunk after this segment
+    bool first;        // first segment of its chunk
+    uint32_t n0;       // stages of this CTA before the segment (ring positions derive from it)
+    __device__ __forceinline__ SegWalk(const TileParams& p_)
+        : p(p_), ci((int)blockIdx.x), t(0), nt(0), mt_i(0), g0(0), units(0), left(0), first(true), n0(0) {
+        load_chunk();
     }
-    __device__ __forceinline__ void load() {
+    __device__ __forceinline__ void load_chunk() {
         long long u0 = 0;
+        int len = 0;
         while (ci < p.nchunks) {
             u0 = tile_chunk_begin(p, ci);
-            left = (int)(tile_chunk_begin(p, ci + 1) - u0);
-            if (left > 0) break;
+            len = (int)(tile_chunk_begin(p, ci + 1) - u0);
+            if (len > 0) break;
             ci += (int)gridDim.x;
         }
-        t0 = t = (int)(u0 / p.G);
-        g0 = g = (int)(u0 - (long long)t * p.G);
+        if (ci >= p.nchunks) return;
+        t = (int)(u0 / p.G);
+        g0 = (int)(u0 - (long long)t * p.G);
         mt_i = t / p.n_tiles;
         nt = t - mt_i * p.n_tiles;
-        c = 0;
-        first_unit = true;
+        units = min(len, p.G - g0);
+        left = len - units;
+        first = true;
     }
     __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
     __device__ __forceinline__ void next() {
-        ++n;
-        if (++slot == stages) { slot = 0; ph ^= 1u; }
-        if (c == 0) { c = 1; return; }
-        c = 0;
-        if (--left == 0) { ci += (int)gridDim.x; load(); return; }
-        first_unit = false;
-        if (++g == p.G) {
-            g = 0;
-            ++t;
-            if (++nt == p.n_tiles) { nt = 0; ++mt_i; }
+        n0 += 2u * (uint32_t)units;
+        if (left == 0) {
+            ci += (int)gridDim.x;
+            load_chunk();
+            return;
         }
+        ++t;
+        if (++nt == p.n_tiles) { nt = 0; ++mt_i; }
+        g0 = 0;
+        units = min(left, p.G);
+        left -= units;
+        first = false;
     }
-    // first / last stage of a segment (the part of the chunk inside one tile)
-    __device__ __forceinline__ bool seg_first() const { return c == 0 && (g == 0 || first_unit); }
-    __device__ __forceinline__ bool seg_last() const { return c == 1 && (g == p.G - 1 || left == 1); }
-    // does the segment of the current stage start at the chunk's first unit / at the tile's first group
-    __device__ __forceinline__ bool seg_starts_chunk() const { return t == t0; }
-    __device__ __forceinline__ bool seg_starts_tile() const { return t != t0 || g0 == 0; }
+    __device__ __forceinline__ int stages_in_seg() const { return 2 * units; }
+    __device__ __forceinline__ bool whole_tile() const { return g0 == 0 && units == p.G; }
+};
+
+// Position in the ring of R slots: slot = n % R, phase = (n / R) & 1, kept incrementally.
+struct RingPos {
+    int slot;
+    uint32_t ph;
+    __device__ __forceinline__ void advance(int d, int R) {
+        slot += d;
+        while (slot >= R) { slot -= R; ph ^= 1u; }
+    }
 };
 
 // Packed words, scale and zero point of one thread's column for one 64-k stage.
@@ -264,9 +271,8 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     constexpr int kDBufs = MT <= 128 ? 2 : 1;            // accumulators in TMEM
     constexpr int kDStride = 128;                        // column distance between the two
 
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [R]  activation box landed
-    uint64_t* a_full = full + kTileMaxStages;                    // [R]  dequantized operand stored in TMEM
-    uint64_t* retired = a_full + kTileMaxStages;                 // [R]  the stage's MMAs retired: slot free
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [R]  activation box landed AND operand stored in TMEM
+    uint64_t* retired = full + kTileMaxStages;                   // [R]  the stage's MMAs retired: slot free
     uint64_t* d_full = retired + kTileMaxStages;                 // [2]  accumulator complete
     uint64_t* d_empty = d_full + 2;                              // [2]  accumulator drained by the epilogue
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(d_empty + 2);
@@ -274,12 +280,11 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     unsigned char* stage0 = smem + kTileBarBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int stages = p.stages;
+    const int R = p.stages;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < stages; ++i) {
-            mbar_init(&full[i], 1);
-            mbar_init(&a_full[i], 4);
+        for (int i = 0; i < R; ++i) {
+            mbar_init(&full[i], 1 + 4);      // the producer's arrive.expect_tx + one arrival per warp of a dequant set
             mbar_init(&retired[i], 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -309,19 +314,26 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         if (elect_one()) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         asm volatile("griddepcontrol.wait;" ::: "memory");   // activations may come from the previous kernel
         bool ok = true;
-        StageWalk w(p);
-        for (; w.valid(); w.next()) {
-            const int slot = w.slot;
-            if (w.n >= (uint32_t)stages && !mbar_wait(&retired[slot], w.ph ^ 1u)) { ok = false; break; }
-            if (elect_one()) {
-                mbar_expect_tx(&full[slot], (uint32_t)MT * 128u);
-                tma_load_2d(stage0 + (size_t)slot * kStageBytes, &tmap_a, w.g * kGroup + w.c * kTileStageK, w.mt_i * MT,
-                            &full[slot]);
+        RingPos r{0, 0u};
+        uint32_t n = 0;
+        for (SegWalk w(p); w.valid() && ok; w.next()) {
+            int k = w.g0 * kGroup;
+            const int m = w.mt_i * MT;
+            const int nst = w.stages_in_seg();
+            for (int j = 0; j < nst; ++j) {
+                if (n >= (uint32_t)R && !mbar_wait(&retired[r.slot], r.ph ^ 1u)) { ok = false; break; }
+                if (elect_one()) {
+                    mbar_expect_tx(&full[r.slot], (uint32_t)MT * 128u);
+                    tma_load_2d(stage0 + (size_t)r.slot * kStageBytes, &tmap_a, k, m, &full[r.slot]);
+                }
+                __syncwarp();
+                k += kTileStageK;
+                ++n;
+                r.advance(1, R);
             }
-            __syncwarp();
         }
         if (lane == 0) {
-            flags[1] = (int)w.n;
+            flags[1] = (int)n;
             if (!ok) *abort_flag = 1;
         }
     } else if (warp == 1) {
@@ -329,37 +341,36 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         asm volatile("griddepcontrol.wait;" ::: "memory");
         uint32_t n_seg = 0;
         bool ok = true;
-        for (StageWalk w(p); w.valid(); w.next()) {
-            const int slot = w.slot;
+        RingPos r{0, 0u};
+        for (SegWalk w(p); w.valid() && ok; w.next(), ++n_seg) {
             const int dbuf = n_seg % kDBufs;
-            const bool first = w.seg_first();
-            if (first) {
-                // the epilogue of the segment that used this accumulator before must have drained it
-                if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
-            }
-            if (!mbar_wait(&full[slot], w.ph) || !mbar_wait(&a_full[slot], w.ph)) { ok = false; break; }
-            tc_fence_after();
-            const bool last = w.seg_last();
-            if (elect_one()) {
-                const uint64_t bdesc = smem_desc_sw128(smem_u32(stage0 + (size_t)slot * kStageBytes));
-                const uint32_t a_t = tmem_base + kTileAColBase + slot * 32;
-                const uint32_t d_t = tmem_base + dbuf * kDStride;
+            // the epilogue of the segment that used this accumulator before must have drained it
+            if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
+            const uint32_t d_t = tmem_base + dbuf * kDStride;
+            const int nst = w.stages_in_seg();
+            for (int j = 0; j < nst; ++j) {
+                if (!mbar_wait(&full[r.slot], r.ph)) { ok = false; break; }
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(stage0 + (size_t)r.slot * kStageBytes));
+                    const uint32_t a_t = tmem_base + kTileAColBase + r.slot * 32;
 #pragma unroll
-                for (int kk = 0; kk < kTileStageK / 16; ++kk) {
-                    // 16 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled rows of B
-                    tc_mma_ts(d_t, a_t + kk * 8, bdesc + (uint64_t)(kk * 2), kIdesc, (first && kk == 0) ? 0u : 1u);
+                    for (int kk = 0; kk < kTileStageK / 16; ++kk) {
+                        // 16 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled rows of B
+                        tc_mma_ts(d_t, a_t + kk * 8, bdesc + (uint64_t)(kk * 2), kIdesc, (j == 0 && kk == 0) ? 0u : 1u);
+                    }
+                    tc_commit(&retired[r.slot]);
+                    if (j == nst - 1) tc_commit(&d_full[dbuf]);
                 }
-                tc_commit(&retired[slot]);
-                if (last) tc_commit(&d_full[dbuf]);
+                __syncwarp();
+                r.advance(1, R);
             }
-            __syncwarp();
-            if (last) ++n_seg;
         }
         if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------ dequant + epilogue warps
         const int dw = warp - 2;               // 0..15
-        const int set = dw >> 2;               // stages with (index % 4) == set
+        const int set = dw >> 2;               // takes the stages whose index in this CTA is = set (mod 4)
         const int quarter = warp & 3;          // TMEM lanes this warp may touch
         const int row = quarter * 32 + lane;   // column n inside the CTA tile = TMEM lane
         const int half = row >> 6, col = row & 63;
@@ -369,12 +380,14 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         const int wo1 = (col >> 3) * 64 + 32 + (((col & 7) + 4) & 7) * 4;
         const int zsh = 4 * (col & 7);
 
-        // packed words of the stage the load walker stands on (zeros past the matrix edge)
-        auto load_stage = [&](const StageWalk& w, StageRegs& r) {
+        // this set's first stage inside a segment
+        auto first_own = [&](const SegWalk& w) { return (int)(((uint32_t)set - w.n0) & 3u); };
+        // packed words of stage j of the load walker's segment (zeros past the matrix edge)
+        auto load_stage = [&](const SegWalk& w, int j, StageRegs& r) {
             const int t64 = 2 * w.nt + half;                      // 64-column packed tile
             if (t64 * kTileN < p.N) {
-                const size_t blk = (size_t)t64 * p.G + w.g;
-                const uint32_t* wp = p.Wq + blk * kBlockWords + w.c * 512;
+                const size_t blk = (size_t)t64 * p.G + (w.g0 + (j >> 1));
+                const uint32_t* wp = p.Wq + blk * kBlockWords + (j & 1) * 512;
                 r.w0 = __ldg(reinterpret_cast<const uint4*>(wp + wo0));
                 r.w1 = __ldg(reinterpret_cast<const uint4*>(wp + wo1));
                 r.s = __ldg(reinterpret_cast<const unsigned short*>(p.S) + blk * kSBlockHalves + col);
@@ -386,45 +399,53 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 r.zw = 0;
             }
         };
-        // advance a walker to this set's next stage at or after its position
-        auto seek_own = [&](StageWalk& w) {
-            while (w.valid() && (int)(w.n % kTileSets) != set) w.next();
-        };
 
+        // load cursor: runs kTilePrefetch of this set's stages ahead of the compute loop
+        SegWalk wl(p);
+        int jl = wl.valid() ? first_own(wl) : 0;
+        auto settle = [&]() {   // move the cursor to a segment that still has a stage of this set
+            while (wl.valid() && jl >= wl.stages_in_seg()) {
+                wl.next();
+                if (wl.valid()) jl = first_own(wl);
+            }
+        };
+        settle();
         StageRegs pf[kTilePrefetch];
-        StageWalk wl(p);
-        seek_own(wl);
 #pragma unroll
         for (int i = 0; i < kTilePrefetch; ++i) {
             if (wl.valid()) {
-                load_stage(wl, pf[i]);
-                wl.next();
-                seek_own(wl);
+                load_stage(wl, jl, pf[i]);
+                jl += kTileSets;
+                settle();
             }
         }
         // everything below may read or write memory the previous kernel is still writing
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
-        uint32_t n_seg = 0;
+        uint32_t n_seg = 0, n_prev = 0;
+        RingPos rp{0, 0u};
         bool ok = true;
-        for (StageWalk w(p); w.valid() && ok; w.next()) {
-            if ((int)(w.n % kTileSets) == set) {
-                const int slot = w.slot;
+        for (SegWalk w(p); w.valid() && ok; w.next(), ++n_seg) {
+            const int nst = w.stages_in_seg();
+            for (int j = first_own(w); j < nst; j += kTileSets) {
+                const uint32_t n = w.n0 + (uint32_t)j;
+                rp.advance((int)(n - n_prev), R);
+                n_prev = n;
                 const StageRegs cur = pf[0];
 #pragma unroll
                 for (int i = 0; i + 1 < kTilePrefetch; ++i) pf[i] = pf[i + 1];
                 if (wl.valid()) {
-                    load_stage(wl, pf[kTilePrefetch - 1]);
-                    wl.next();
-                    seek_own(wl);
+                    load_stage(wl, jl, pf[kTilePrefetch - 1]);
+                    jl += kTileSets;
+                    settle();
                 }
                 const uint32_t z = (cur.zw >> zsh) & 15u;
                 const __half2 s2 = u32_as_h2(cur.s * 0x00010001u);
                 const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
                 // the MMAs that read this slot one ring turn ago must have retired
-                if (w.n >= (uint32_t)stages && !mbar_wait(&retired[slot], w.ph ^ 1u)) { ok = false; break; }
+                if (n >= (uint32_t)R && !mbar_wait(&retired[rp.slot], rp.ph ^ 1u)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_t = tmem_base + lane_addr + kTileAColBase + slot * 32;
+                const uint32_t a_t = tmem_base + lane_addr + kTileAColBase + rp.slot * 32;
                 {
                     const uint32_t ww[4] = {cur.w0.x, cur.w0.y, cur.w0.z, cur.w0.w};   // k = 0 .. 31
                     uint32_t regs[16];
@@ -432,7 +453,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                     for (int i = 0; i < 4; ++i) {
                         const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) regs[4 * i + j] = h2_as_u32(f.h[j]);
+                        for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
                     }
                     tc_st16(a_t, regs);
                 }
@@ -443,31 +464,29 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                     for (int i = 0; i < 4; ++i) {
                         const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) regs[4 * i + j] = h2_as_u32(f.h[j]);
+                        for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
                     }
                     tc_st16(a_t + 16, regs);
                 }
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[slot]);
+                if (lane == 0) mbar_arrive(&full[rp.slot]);
             }
-            if (!w.seg_last()) continue;
+            if (!ok) break;
 
-            // ---------------------------------------------------- epilogue of the segment that ends here
+            // ---------------------------------------------------- epilogue of this segment
             const int dbuf = n_seg % kDBufs;
             if (!mbar_wait(&d_full[dbuf], (n_seg / kDBufs) & 1u)) { ok = false; break; }
-            ++n_seg;
             tc_fence_after();
             const int T = w.t;
-            const int nt = w.nt, mt_i = w.mt_i;
-            const int n = nt * kTileCols + row;
-            const int m_base = mt_i * MT + set * kCW;     // first batch row of this warp's columns
+            const int n = w.nt * kTileCols + row;
+            const int m_base = w.mt_i * MT + set * kCW;     // first batch row of this warp's columns
             const uint32_t d_t = tmem_base + lane_addr + dbuf * kDStride + set * kCW;
             const long long tile_u0 = (long long)T * p.G;
-            const bool whole = w.seg_starts_tile() && (w.g == p.G - 1);
+            const bool whole = w.whole_tile();
             // first segment of a chunk -> slot 2 ci, its continuation into a later tile -> 2 ci + 1
-            float* part = p.ws + ((size_t)(2 * w.ci + (w.seg_starts_chunk() ? 0 : 1)) * MT + set * kCW) * kTileCols + row;
+            float* part = p.ws + ((size_t)(2 * w.ci + (w.first ? 0 : 1)) * MT + set * kCW) * kTileCols + row;
             constexpr int kStep = kCW >= 16 ? 16 : kCW;
 #pragma unroll 1
             for (int cc = 0; cc < kCW; cc += kStep) {
@@ -479,14 +498,14 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 if (whole) {
                     if (n < p.N) {
 #pragma unroll
-                        for (int j = 0; j < kStep; ++j) {
-                            const int m = m_base + cc + j;
-                            if (m < p.M) p.C[(size_t)m * p.N + n] = __float2half_rn(__uint_as_float(v[j]));
+                        for (int q = 0; q < kStep; ++q) {
+                            const int m = m_base + cc + q;
+                            if (m < p.M) p.C[(size_t)m * p.N + n] = __float2half_rn(__uint_as_float(v[q]));
                         }
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < kStep; ++j) part[(size_t)(cc + j) * kTileCols] = __uint_as_float(v[j]);
+                    for (int q = 0; q < kStep; ++q) part[(size_t)(cc + q) * kTileCols] = __uint_as_float(v[q]);
                 }
             }
             // accumulator drained: a later segment's first MMA may overwrite it
@@ -511,17 +530,29 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 if (last) {
                     __threadfence();
                     // contributors in ascending K: chunk c_first (its first segment if it starts at the tile's
-                    // first unit, else its continuation), then the first segments of the others
+                    // first unit, else its continuation), then the first segments of the others.  Rows are
+                    // summed kStep at a time so that many loads are in flight.
                     const size_t slot_elems = (size_t)MT * kTileCols;
                     const float* base = p.ws + (size_t)(set * kCW) * kTileCols + row;
                     const size_t first_slot = 2 * (size_t)c_first + (tile_chunk_begin(p, c_first) == tile_u0 ? 0 : 1);
-#pragma unroll 2
-                    for (int mm = 0; mm < kCW; ++mm) {
-                        float acc = __ldcg(base + first_slot * slot_elems + (size_t)mm * kTileCols);
-                        for (int c = c_first + 1; c <= c_last; ++c)
-                            acc += __ldcg(base + (size_t)(2 * c) * slot_elems + (size_t)mm * kTileCols);
-                        const int m = m_base + mm;
-                        if (m < p.M && n < p.N) p.C[(size_t)m * p.N + n] = __float2half_rn(acc);
+#pragma unroll 1
+                    for (int m0 = 0; m0 < kCW; m0 += kStep) {
+                        float acc[kStep];
+#pragma unroll
+                        for (int q = 0; q < kStep; ++q)
+                            acc[q] = __ldcg(base + first_slot * slot_elems + (size_t)(m0 + q) * kTileCols);
+                        for (int c = c_first + 1; c <= c_last; ++c) {
+                            const float* src = base + (size_t)(2 * c) * slot_elems + (size_t)m0 * kTileCols;
+#pragma unroll
+                            for (int q = 0; q < kStep; ++q) acc[q] += __ldcg(src + (size_t)q * kTileCols);
+                        }
+                        if (n < p.N) {
+#pragma unroll
+                            for (int q = 0; q < kStep; ++q) {
+                                const int m = m_base + m0 + q;
+                                if (m < p.M) p.C[(size_t)m * p.N + n] = __float2half_rn(acc[q]);
+                            }
+                        }
                     }
                 }
             }
@@ -534,11 +565,12 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     __syncthreads();
     if (*abort_flag != 0 && threadIdx.x == 0) {
         // some wait ran out: before the CTA's shared memory goes away, give the copies still in
-        // flight a (bounded) chance to land -- the last use of every stage slot
+        // flight a (bounded) chance to land -- the last use of every ring slot.  (The phase may lack
+        // the dequant warps' arrivals and then runs into the limit; the wait is bounded either way.)
         const uint32_t issued = (uint32_t)flags[1];
-        for (uint32_t back = 0; back < (uint32_t)stages && back < issued; ++back) {
+        for (uint32_t back = 0; back < (uint32_t)R && back < issued; ++back) {
             const uint32_t ns = issued - 1 - back;
-            mbar_wait(&full[ns % stages], (ns / stages) & 1u);
+            mbar_wait(&full[ns % R], (ns / R) & 1u);
         }
     }
     __syncthreads();
