@@ -33,10 +33,12 @@ UNIT = "GB/s"
 SWEEP_K, SWEEP_N, SWEEP_M = 11008, 4096, (1, 2, 4, 8, 16)
 WORKLOAD = "config2_down_proj_decode_K11008_N4096_M1-2-4-8-16"
 MIN_ROTATION_BYTES = 512 << 20
+PATH_NAMES = {1: "gemm_simple_kernel", 2: "gemm_decode_kernel", 3: "gemm_tile_kernel"}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until captured)
 NCU_TRAFFIC_BYTES = None
+NCU_TRAFFIC_BYTES_TILE = None
 
 
 def _peaks():
@@ -235,6 +237,8 @@ def run_ours(args):
     if args.configs:
         for c in wl.CASES:
             if c.config in args.configs and not (c.config == 2):
+                if world > 1 and c.config != 2:
+                    continue        # the per-case table is a 1-GPU report
                 extra_cases.append(c)
         for c in extra_cases:
             ws_need = max(ws_need, B.w4a16_workspace_bytes(c.M, c.N, c.K, 128, 0))
@@ -300,6 +304,7 @@ def run_ours(args):
         byts = wl.algorithmic_bytes(M, K, N)
         per_call[M] = sec
         cases.append({"config": 2, "layer": "down_proj", "M": M, "K": K, "N": N, "split_k": splits[i],
+                      "path": PATH_NAMES.get(B.w4a16_choose_path(M, N, K), "?"),
                       "us": sec * 1e6, "eff_GBps": byts / sec / 1e9, "tflops": 2.0 * M * N * K / sec / 1e12,
                       "roofline_frac": max(byts / (hbm_peak * 1e9), 2.0 * M * N * K / (tc_peak * 1e12)) / sec})
     # split_k = 1 ("data parallel" in the paper's comparison) beside the chosen split
@@ -324,9 +329,11 @@ def run_ours(args):
 
     # other configs on request (each case alone, rotating copies)
     cur = None
+    cur_w16 = None
     for c in extra_cases:
         if cur is None or (cur.K, cur.N) != (c.K, c.N):
             cur = None
+            cur_w16 = None
             torch.cuda.empty_cache()
             cur = Layer(c.K, c.N, c.seed, torch, B, wl)
         A = _to_dev(wl.draw_activations(c.M, c.K, c.seed, c.a_sigma, c.outliers), torch)
@@ -336,9 +343,24 @@ def run_ours(args):
                           max(20, args.case_calls // 4), torch)
         byts = wl.algorithmic_bytes(c.M, c.K, c.N)
         fl = 2.0 * c.M * c.N * c.K
-        cases.append({"config": c.config, "layer": c.name, "M": c.M, "K": c.K, "N": c.N, "split_k": s,
-                      "us": sec * 1e6, "eff_GBps": byts / sec / 1e9, "tflops": fl / sec / 1e12,
-                      "roofline_frac": max(byts / (hbm_peak * 1e9), fl / (tc_peak * 1e12)) / sec})
+        rec = {"config": c.config, "layer": c.name, "M": c.M, "K": c.K, "N": c.N, "split_k": s,
+               "path": PATH_NAMES.get(B.w4a16_choose_path(c.M, c.N, c.K), "?"),
+               "us": sec * 1e6, "eff_GBps": byts / sec / 1e9, "tflops": fl / sec / 1e12,
+               "bound": "tensor" if fl / (tc_peak * 1e12) > byts / (hbm_peak * 1e9) else "hbm",
+               "roofline_frac": max(byts / (hbm_peak * 1e9), fl / (tc_peak * 1e12)) / sec}
+        if not args.no_cublas:
+            if cur_w16 is None:
+                ncopy = max(2, min(6, (MIN_ROTATION_BYTES // 2) // (c.K * c.N * 2) + 1))
+                cur_w16 = [B.w4a16_dequant(cur.packed[0]).clone() for _ in range(ncopy)]
+            k16 = [0]
+
+            def mm16():
+                torch.matmul(A, cur_w16[k16[0] % len(cur_w16)], out=C)
+                k16[0] += 1
+            sec16 = _time_calls(mm16, 5, max(20, args.case_calls // 8), torch, per_graph=8)
+            rec["torch_fp16_matmul_us"] = sec16 * 1e6
+            rec["speedup_vs_fp16"] = sec16 / sec
+        cases.append(rec)
 
     # ---- end to end through the host-buffer entry point (H2D of A and D2H of C inside the region)
     hA = [torch.from_numpy(a.view(np.float16)).pin_memory() for a in acts_np]
@@ -368,7 +390,7 @@ def run_ours(args):
     dom_M = SWEEP_M[-1]
     dom_bytes = wl.algorithmic_bytes(dom_M, K, N)
     achieved = dom_bytes / per_call[dom_M] / 1e9
-    roofline = {"bound": "hbm", "kernel": "gemm_decode_kernel", "case": "M=%d K=%d N=%d" % (dom_M, K, N),
+    roofline = {"bound": "hbm", "kernel": PATH_NAMES.get(B.w4a16_choose_path(dom_M, N, K), "?"), "case": "M=%d K=%d N=%d" % (dom_M, K, N),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                 "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES,
                 "algorithmic_bytes_per_launch": dom_bytes,
@@ -394,6 +416,29 @@ def run_ours(args):
                "sample": "%d full steps (all 5 GEMMs, all columns), %.1f s of CPU time" % (reps_cpu, dt),
                "max_elem_err_vs_gpu": worst}
 
+    # the tensor-bound end of the path: the largest prefill case that was timed (config 5)
+    roofline_tensor = None
+    big = [c for c in cases if c["config"] == 5]
+    if big:
+        b = max(big, key=lambda c: c["M"])
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except Exception:
+            pass
+        sustained = float(peaks.get("bf16_tflops_sustained", 1400.0))
+        roofline_tensor = {"bound": "tensor", "kernel": b["path"], "case": "M=%d K=%d N=%d" % (b["M"], b["K"], b["N"]),
+                           "achieved": b["tflops"], "peak": tc_peak, "peak_kind": "of " + peak_kind +
+                           " (burst; FP16 takes the BF16 figure, same nominal rate)", "unit": "TFLOP/s",
+                           "frac": b["tflops"] / tc_peak, "frac_of_sustained_peak": b["tflops"] / sustained,
+                           "launch_us": b["us"], "traffic": NCU_TRAFFIC_BYTES_TILE}
+    # config 4: the four layers of one transformer block, summed per batch size
+    block_sums = {}
+    for c in cases:
+        if c["config"] == 4:
+            block_sums.setdefault(c["M"], 0.0)
+            block_sums[c["M"]] += c["us"]
+
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -413,6 +458,8 @@ def run_ours(args):
                             "packed weights resident in HBM"},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline,
+            "roofline_tensor": roofline_tensor,
+            "config4_block_us_by_M": block_sums,
             "cpu_baseline": cpu,
             "cases": cases,
         }))
@@ -466,8 +513,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--split-k", type=int, default=0, help="force one split factor (0 = automatic)")
-    ap.add_argument("--configs", type=lambda s: [int(x) for x in s.split(",")], default=None,
-                    help="also time every case of these configs (e.g. 1,3,4,5)")
+    ap.add_argument("--configs", type=lambda s: [int(x) for x in s.split(",")], default=[1, 3, 4, 5],
+                    help="besides the timed config-2 step, report every case of these configs (2 = none)")
     ap.add_argument("--case-calls", type=int, default=400)
     ap.add_argument("--no-cublas", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -94,6 +94,8 @@ int w4a16_set_workspace(void *dev_ptr, size_t bytes);
  * w4a16_gemm accepts; >= 1.  `path` as in w4a16_gemm_ex. */
 int w4a16_choose_split_k(int M, int N, int K, int group);
 int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path);
+/* The kernel path (W4A16_PATH_*) w4a16_gemm takes for a shape, or a negative error code. */
+int w4a16_choose_path(int M, int N, int K, int group);
 
 /* Offline reorder of the raw nibbles, scales and zero points into the packed layout
  * (pure data movement, a bijection; Section 2.2 storage packing).  Reads the three raw

@@ -24,7 +24,7 @@ WS_HEADER_BYTES = 16384 + 131072   # W4A16_WORKSPACE_HEADER_BYTES
 EXPORTS = (
     "w4a16_strerror", "w4a16_packed_wq_bytes", "w4a16_packed_s_bytes", "w4a16_packed_z_bytes",
     "w4a16_workspace_bytes", "w4a16_set_workspace", "w4a16_choose_split_k",
-    "w4a16_choose_split_k_ex", "w4a16_pack", "w4a16_dequant", "w4a16_gemm", "w4a16_gemm_ex",
+    "w4a16_choose_split_k_ex", "w4a16_choose_path", "w4a16_pack", "w4a16_dequant", "w4a16_gemm", "w4a16_gemm_ex",
     "w4a16_gemm_host", "w4a16_gemm_static_ws", "w4a16_device_status",
 )
 
@@ -59,6 +59,8 @@ def load():
     L.w4a16_set_workspace.argtypes = [vp, sz]
     L.w4a16_choose_split_k.restype = i
     L.w4a16_choose_split_k.argtypes = [i, i, i, i]
+    L.w4a16_choose_path.restype = i
+    L.w4a16_choose_path.argtypes = [i, i, i, i]
     L.w4a16_choose_split_k_ex.restype = i
     L.w4a16_choose_split_k_ex.argtypes = [i, i, i, i, i]
     L.w4a16_pack.restype = i
@@ -115,6 +117,10 @@ def w4a16_workspace_bytes(M: int, N: int, K: int, group: int = GROUP, split_k: i
 
 def w4a16_choose_split_k(M: int, N: int, K: int, group: int = GROUP, path: int = PATH_AUTO) -> int:
     return load().w4a16_choose_split_k_ex(M, N, K, group, path)
+
+
+def w4a16_choose_path(M: int, N: int, K: int, group: int = GROUP) -> int:
+    return load().w4a16_choose_path(M, N, K, group)
 
 
 def w4a16_set_workspace(ws: Optional[torch.Tensor]) -> None:

@@ -279,6 +279,10 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
         default: return 1;
     }
 }
+int w4a16_choose_path(int M, int N, int K, int group) {
+    if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return W4A16_ERR_SHAPE;
+    return resolve_path(M, W4A16_PATH_AUTO);
+}
 int w4a16_choose_split_k(int M, int N, int K, int group) {
     return w4a16_choose_split_k_ex(M, N, K, group, W4A16_PATH_AUTO);
 }

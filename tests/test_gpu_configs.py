@@ -1,0 +1,60 @@
+"""GPU parity at the benchmark's full sizes (configs 1-4), in the launch configuration bench.py
+times: automatic path, automatic split.  The oracle (Eq. 2 in FP64) computes whole columns of C,
+sampled at tile edges, a tile interior and the last columns; all rows of the batch are checked."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_16536_b200 import binding as B
+from paper_2601_16536_b200 import workloads as wl
+from gpu_util import assert_close, c_f64, ensure_ws, pack_problem, to_dev
+
+pytestmark = pytest.mark.gpu
+
+_CASES = [c for c in wl.CASES if c.config in (1, 2, 3, 4)]
+_weights = {}
+
+
+def _packed(case):
+    """One packed copy per (K, N, seed of the first case with that layer): cases of a config share
+    shapes but not seeds, so weights are drawn per case; the cache only spares identical repeats."""
+    key = (case.K, case.N, case.seed)
+    if key not in _weights:
+        _weights.clear()
+        d = wl.draw_weights(case.K, case.N, case.seed)
+        _weights[key] = (d, pack_problem(d, case.N, case.K))
+    return _weights[key]
+
+
+@pytest.mark.parametrize("case", _CASES, ids=lambda c: "cfg%d-%s-M%d" % (c.config, c.name, c.M))
+def test_full_size_case_sampled_columns(case):
+    M, K, N = case.M, case.K, case.N
+    d, pw = _packed(case)
+    A_bits = wl.draw_activations(M, K, case.seed, case.a_sigma, case.outliers)
+    ws = ensure_ws(M, N, K, 0)
+    C = B.w4a16_gemm(to_dev(A_bits), pw)
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    got = c_f64(C)
+    assert np.all(np.isfinite(got))
+    for n0 in (0, 62, 127, N // 2 - 3, N - 4):
+        ref = oracle.gemm(A_bits, d["Wq"], d["S"], d["Z"], M, N, K, 128, cols=(n0, n0 + 4))
+        assert_close(got[:, n0:n0 + 4], ref[:, n0:n0 + 4], "cfg%d %s M%d cols %d" % (case.config, case.name, M, n0))
+    del ws
+
+
+def test_results_do_not_depend_on_the_path():
+    # the same product through the plain, the warp-MMA and the tcgen05 kernels: each within
+    # tolerance of the oracle, hence of each other
+    M, K, N = 16, 2048, 1024
+    d = wl.make_problem(M, K, N, seed=4711)
+    pw = pack_problem(d, N, K)
+    A = to_dev(d["A"])
+    ws = ensure_ws(M, N, K, 0)
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+    for path in (B.PATH_SIMPLE, B.PATH_DECODE, B.PATH_TILE, B.PATH_AUTO):
+        C = B.w4a16_gemm(A, pw, path=path)
+        torch.cuda.synchronize()
+        assert_close(c_f64(C), ref, "path %d" % path)
+    del ws
