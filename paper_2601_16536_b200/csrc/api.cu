@@ -482,9 +482,24 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
         }
         d->decode_attr_set[g.mb] = true;
     }
-    dim3 grid(g.ctas, g.mchunks, 1);
-    kern<<<grid, kDecThreads, g.smem_bytes, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
+    // programmatic dependent launch (see the tile path above): prologue and weight prefetch may overlap
+    // the tail of the previous kernel in the stream
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(g.ctas, g.mchunks, 1);
+    cfg.blockDim = dim3(kDecThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = d->pdl_ok ? 1 : 0;
+    d->pdl_ok = true;
+    if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) {
+        cudaGetLastError();
+        return W4A16_ERR_CUDA;
+    }
+    return W4A16_OK;
 }
 
 int w4a16_gemm(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,

@@ -96,6 +96,33 @@ __device__ __forceinline__ int chunk_of(const DecodeParams& p, int u) {
     return t * p.split_k + s;
 }
 
+// The stages of a CTA in order: up to four consecutive units of one tile each.
+struct DecStageIter {
+    const DecodeParams& p;
+    int ci, u, u1, t, tile_end;
+    __device__ __forceinline__ DecStageIter(const DecodeParams& p_) : p(p_), ci((int)blockIdx.x), u(0), u1(0), t(0), tile_end(0) {
+        load();
+    }
+    __device__ __forceinline__ void load() {
+        while (ci < p.nchunks) {
+            u = chunk_begin(p, ci);
+            u1 = chunk_begin(p, ci + 1);
+            if (u < u1) break;
+            ci += (int)gridDim.x;
+        }
+        t = u / p.G;
+        tile_end = (t + 1) * p.G;
+    }
+    __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
+    __device__ __forceinline__ int units() const { return min(kDecUnitsPerStage, min(u1, tile_end) - u); }
+    __device__ __forceinline__ int group() const { return u - t * p.G; }
+    __device__ __forceinline__ void next() {
+        u += units();
+        if (u == tile_end) { ++t; tile_end += p.G; }
+        if (u >= u1) { ci += (int)gridDim.x; load(); }
+    }
+};
+
 // MB = number of 8-row batch blocks one CTA handles (rows m0 .. m0 + 8 MB - 1).
 template <int MB>
 __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodeParams p) {
@@ -122,61 +149,63 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
         }
         fence_mbar_init();
     }
-    // activation rows this CTA does not have stay zero for the whole kernel
-    if (rows < kRows) {
-        for (int s = 0; s < stages; ++s) {
-            uint32_t* z = reinterpret_cast<uint32_t*>(stage0 + (size_t)s * stage_bytes + kDecStageA +
-                                                      rows * kDecARowBytes);
-            for (int i = threadIdx.x; i < (kRows - rows) * kDecARowBytes / 4; i += kDecThreads) z[i] = 0u;
-        }
-    }
+    // (Batch rows this CTA does not have are never loaded: an MMA column only feeds its own output
+    // column, and those columns are not stored.)
     __syncthreads();
-    // Let the next kernel in the stream start its own prologue; everything below that reads
-    // or writes memory another kernel may have written comes after griddepcontrol.wait.
+    // Let the next kernel in the stream start its own prologue and weight prefetch; everything below
+    // that reads or writes memory another kernel may have written comes after griddepcontrol.wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kDecWarps) {
         // ------------------------------------------------ producer warp
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        int slot = 0;
-        uint32_t phase = 0;
-        bool first_round = true;
-        for (int ci = blockIdx.x; ci < p.nchunks; ci += gridDim.x) {
-            int u = chunk_begin(p, ci);
-            const int u1 = chunk_begin(p, ci + 1);
-            if (u >= u1) continue;
-            int t = u / p.G;
-            int tile_end = (t + 1) * p.G;
-            while (u < u1) {
-                const int gc = min(kDecUnitsPerStage, min(u1, tile_end) - u);
-                if (!first_round) {
-                    if (!mbar_wait(&empty[slot], phase ^ 1u)) return;  // status recorded
+        auto issue_weights = [&](const DecStageIter& it, unsigned char* st, uint64_t* bar, int gc) {
+            bulk_g2s(st, p.Wq + (size_t)it.u * kBlockWords, (uint32_t)(gc * kBlockBytes), bar);
+            bulk_g2s(st + kDecStageS, p.S + (size_t)it.u * kSBlockHalves, (uint32_t)(gc * kSBlockHalves * 2), bar);
+            bulk_g2s(st + kDecStageZ, p.Z + (size_t)it.u * kZBlockWords, (uint32_t)(gc * kZBlockWords * 4), bar);
+        };
+        auto issue_rows = [&](const DecStageIter& it, unsigned char* st, uint64_t* bar, int gc) {
+            const int g = it.group();  // the stage's units are groups g .. g + gc - 1 of tile t
+            for (int m = lane; m < rows; m += 32) {
+                bulk_g2s(st + kDecStageA + m * kDecARowBytes, p.A + (size_t)(m0 + m) * p.K + (size_t)g * kGroup,
+                         (uint32_t)(gc * kGroup * 2), bar);
+            }
+        };
+        // 1. packed weights of the first ring-full of stages: they do not depend on the previous kernel
+        {
+            DecStageIter pre(p);
+            for (int i = 0; i < stages && pre.valid(); ++i, pre.next()) {
+                if (lane == 0) {
+                    const int gc = pre.units();
+                    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full[i])),
+                                 "r"((uint32_t)(gc * kDecUnitBytes))
+                                 : "memory");
+                    issue_weights(pre, stage0 + (size_t)i * stage_bytes, &full[i], gc);
                 }
-                unsigned char* st = stage0 + (size_t)slot * stage_bytes;
+            }
+        }
+        // 2. the activations may be the previous kernel's output
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        int slot = 0, n = 0;
+        uint32_t phase = 0;
+        for (DecStageIter it(p); it.valid(); it.next(), ++n) {
+            const int gc = it.units();
+            unsigned char* st = stage0 + (size_t)slot * stage_bytes;
+            if (n < stages) {
+                if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)(rows * gc * (kGroup * 2)));
+                __syncwarp();
+                issue_rows(it, st, &full[slot], gc);
+            } else {
+                if (!mbar_wait(&empty[slot], phase ^ 1u)) return;  // status recorded
                 if (lane == 0) {
                     mbar_expect_tx(&full[slot], (uint32_t)(gc * kDecUnitBytes + rows * gc * (kGroup * 2)));
-                    bulk_g2s(st, p.Wq + (size_t)u * kBlockWords, (uint32_t)(gc * kBlockBytes), &full[slot]);
-                    bulk_g2s(st + kDecStageS, p.S + (size_t)u * kSBlockHalves, (uint32_t)(gc * kSBlockHalves * 2),
-                             &full[slot]);
-                    bulk_g2s(st + kDecStageZ, p.Z + (size_t)u * kZBlockWords, (uint32_t)(gc * kZBlockWords * 4),
-                             &full[slot]);
+                    issue_weights(it, st, &full[slot], gc);
                 }
                 __syncwarp();
-                const int g = u - t * p.G;  // the stage's units are groups g .. g + gc - 1 of tile t
-                for (int m = lane; m < rows; m += 32) {
-                    bulk_g2s(st + kDecStageA + m * kDecARowBytes, p.A + (size_t)(m0 + m) * p.K + (size_t)g * kGroup,
-                             (uint32_t)(gc * kGroup * 2), &full[slot]);
-                }
-                u += gc;
-                if (u == tile_end) {
-                    ++t;
-                    tile_end += p.G;
-                }
-                if (++slot == stages) {
-                    slot = 0;
-                    phase ^= 1u;
-                    first_round = false;
-                }
+                issue_rows(it, st, &full[slot], gc);
+            }
+            if (++slot == stages) {
+                slot = 0;
+                phase ^= 1u;
             }
         }
         return;
