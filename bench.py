@@ -57,6 +57,22 @@ def _rank_world():
         int(os.environ.get("LOCAL_RANK", "0"))
 
 
+# ------------------------------------------------------------------------------ ranks
+def max_over_ranks(seconds, dist, device):
+    """The slowest rank's time: replicas run independently, the job is as slow as its slowest rank."""
+    if dist is None:
+        return float(seconds)
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(step_bytes, steps, world, seconds):
+    """Aggregate effective bandwidth in GB/s: every rank moves step_bytes per step (weak scaling)."""
+    return step_bytes * steps * world / seconds / 1e9
+
+
 # ------------------------------------------------------------------------------ clocks
 class ClockSampler:
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -288,12 +304,9 @@ def run_ours(args):
             g_main.replay()
             torch.cuda.synchronize()
     clocks = sampler.stop()
-    if dist:
-        t = torch.tensor([elapsed], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed = float(t.item())
+    elapsed = max_over_ranks(elapsed, dist, "cuda")
     assert B.w4a16_device_status() == 0, "a kernel reported a device-side timeout"
-    value = step_bytes * args.steps * world / elapsed / 1e9
+    value = whole_job_value(step_bytes, args.steps, world, elapsed)
 
     # ---- per-case numbers (each M alone, same rotation)
     cases = []
@@ -380,11 +393,8 @@ def run_ours(args):
         step_e2e()
     torch.cuda.synchronize()
     e2e_elapsed = time.perf_counter() - t0
-    if dist:
-        t = torch.tensor([e2e_elapsed], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_elapsed = float(t.item())
-    e2e_value = step_bytes * args.steps * world / e2e_elapsed / 1e9
+    e2e_elapsed = max_over_ranks(e2e_elapsed, dist, "cuda")
+    e2e_value = whole_job_value(step_bytes, args.steps, world, e2e_elapsed)
 
     # ---- roofline of the dominant kernel (the decode GEMM kernel at M = 16, the heaviest call)
     dom_M = SWEEP_M[-1]
