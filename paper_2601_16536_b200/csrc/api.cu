@@ -159,6 +159,7 @@ TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     const int avail = max_smem - kTileBarBytes - 1024;   // barrier block + alignment slack
     int st = avail / tile_stage_bytes(g.mt);
     if (st > kTileMaxStages) st = kTileMaxStages;
+    if (st > tile_max_slots(g.mt)) st = tile_max_slots(g.mt);   // the ring also lives in tensor memory
     g.stages = st;
     g.smem_bytes = kTileBarBytes + 1024 + st * tile_stage_bytes(g.mt);
     // each CTA takes the SM's whole tensor memory: ask for enough shared memory that two never share an SM
@@ -207,7 +208,7 @@ bool make_act_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mt) 
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTileStageK, (cuuint32_t)mt};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileBoxK, (cuuint32_t)mt};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(A), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

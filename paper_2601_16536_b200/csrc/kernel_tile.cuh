@@ -48,16 +48,22 @@
 namespace w4a16 {
 
 constexpr int kTileCols = 128;                      // n per CTA tile = UMMA M
-constexpr int kTileStageK = 64;                     // k per pipeline stage
+constexpr int kTileBoxK = 64;                       // k per activation TMA box (one 128-byte swizzle row)
+// k per pipeline stage: a whole group for narrow batch tiles (twice the MMAs per barrier round: the
+// issuing lane and the per-stage synchronisation are what bounds them), half a group otherwise
+__host__ __device__ constexpr int tile_stage_k(int mt) { return mt <= 64 ? 128 : 64; }
 constexpr int kTileDequantWarps = 16;               // four sets of four (one warp per TMEM lane quarter)
 constexpr int kTileSets = kTileDequantWarps / 4;
 constexpr int kTileThreads = (2 + kTileDequantWarps) * 32;   // producer, MMA, dequant/epilogue warps
-constexpr int kTileMaxStages = 8;                   // ring slots: activation box + 32 TMEM columns each
-constexpr int kTileAColBase = 256;                  // accumulators in columns [0, 256), the ring in [256, 512)
-constexpr int kTilePrefetch = 3;                    // stages of packed words a dequant thread holds in registers
+constexpr int kTileMaxStages = 8;                   // ring slots: activation boxes + stage_k / 2 TMEM columns each
+// TMEM columns: the accumulators first (two of up to 128 columns, or one of 256), then the operand ring
+__host__ __device__ constexpr int tile_a_col_base(int mt) { return mt <= 64 ? 128 : 256; }
+__host__ __device__ constexpr int tile_max_slots(int mt) { return (512 - tile_a_col_base(mt)) / (tile_stage_k(mt) / 2); }
+// stages of packed words a dequant thread holds in registers (loads issued that far ahead)
+__host__ __device__ constexpr int tile_prefetch(int mt) { return mt <= 64 ? 2 : 3; }
 constexpr int kTileBarBytes = 1024;
 
-__host__ __device__ constexpr int tile_stage_bytes(int mt) { return mt * 128; }
+__host__ __device__ constexpr int tile_stage_bytes(int mt) { return mt * tile_stage_k(mt) * 2; }
 
 struct TileParams {
     const uint32_t* Wq;
@@ -200,8 +206,9 @@ struct SegWalk {
     int left;          // units of the chunk after this segment
     bool first;        // first segment of its chunk
     uint32_t n0;       // stages of this CTA before the segment (ring positions derive from it)
-    __device__ __forceinline__ SegWalk(const TileParams& p_)
-        : p(p_), ci((int)blockIdx.x), t(0), nt(0), mt_i(0), g0(0), units(0), left(0), first(true), n0(0) {
+    const int spu;     // stages per unit (group): 1 or 2
+    __device__ __forceinline__ SegWalk(const TileParams& p_, int spu_)
+        : p(p_), ci((int)blockIdx.x), t(0), nt(0), mt_i(0), g0(0), units(0), left(0), first(true), n0(0), spu(spu_) {
         load_chunk();
     }
     __device__ __forceinline__ void load_chunk() {
@@ -224,7 +231,7 @@ struct SegWalk {
     }
     __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
     __device__ __forceinline__ void next() {
-        n0 += 2u * (uint32_t)units;
+        n0 += (uint32_t)(spu * units);
         if (left == 0) {
             ci += (int)gridDim.x;
             load_chunk();
@@ -237,7 +244,7 @@ struct SegWalk {
         left -= units;
         first = false;
     }
-    __device__ __forceinline__ int stages_in_seg() const { return 2 * units; }
+    __device__ __forceinline__ int stages_in_seg() const { return spu * units; }
     __device__ __forceinline__ bool whole_tile() const { return g0 == 0 && units == p.G; }
 };
 
@@ -251,9 +258,10 @@ struct RingPos {
     }
 };
 
-// Packed words, scale and zero point of one thread's column for one 64-k stage.
+// Packed words, scale and zero point of one thread's column for one stage of 32 * NW k.
+template <int NW>
 struct StageRegs {
-    uint4 w0, w1;     // k = 0..31 and 32..63 of the stage
+    uint4 w[NW];      // w[i]: k = 32 i .. 32 i + 31 of the stage
     uint32_t s;       // FP16 scale bits
     uint32_t zw;      // zero-point word of the column's 8-column block
 };
@@ -269,7 +277,13 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     constexpr uint32_t kIdesc = tile_idesc(MT);
     constexpr int kCW = MT / kTileSets;                  // accumulator columns (batch rows) per epilogue warp
     constexpr int kDBufs = MT <= 128 ? 2 : 1;            // accumulators in TMEM
-    constexpr int kDStride = 128;                        // column distance between the two
+    constexpr int kDStride = MT <= 64 ? 64 : 128;        // column distance between the two
+    constexpr int kStageK = tile_stage_k(MT);            // k per ring slot
+    constexpr int kSPU = kGroup / kStageK;               // stages per unit
+    constexpr int kSlotCols = kStageK / 2;               // TMEM columns of one operand slot
+    constexpr int kACol = tile_a_col_base(MT);
+    constexpr int kNW = kStageK / 32;                    // 16-byte chunks of a thread's column per stage
+    constexpr int kPF = tile_prefetch(MT);
 
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [R]  activation box landed AND operand stored in TMEM
     uint64_t* retired = full + kTileMaxStages;                   // [R]  the stage's MMAs retired: slot free
@@ -316,18 +330,21 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         bool ok = true;
         RingPos r{0, 0u};
         uint32_t n = 0;
-        for (SegWalk w(p); w.valid() && ok; w.next()) {
+        for (SegWalk w(p, kSPU); w.valid() && ok; w.next()) {
             int k = w.g0 * kGroup;
             const int m = w.mt_i * MT;
             const int nst = w.stages_in_seg();
             for (int j = 0; j < nst; ++j) {
                 if (n >= (uint32_t)R && !mbar_wait(&retired[r.slot], r.ph ^ 1u)) { ok = false; break; }
                 if (elect_one()) {
-                    mbar_expect_tx(&full[r.slot], (uint32_t)MT * 128u);
-                    tma_load_2d(stage0 + (size_t)r.slot * kStageBytes, &tmap_a, k, m, &full[r.slot]);
+                    mbar_expect_tx(&full[r.slot], (uint32_t)kStageBytes);
+#pragma unroll
+                    for (int b = 0; b < kStageK / kTileBoxK; ++b)
+                        tma_load_2d(stage0 + (size_t)r.slot * kStageBytes + b * (MT * 128), &tmap_a, k + b * kTileBoxK, m,
+                                    &full[r.slot]);
                 }
                 __syncwarp();
-                k += kTileStageK;
+                k += kStageK;
                 ++n;
                 r.advance(1, R);
             }
@@ -342,7 +359,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         uint32_t n_seg = 0;
         bool ok = true;
         RingPos r{0, 0u};
-        for (SegWalk w(p); w.valid() && ok; w.next(), ++n_seg) {
+        for (SegWalk w(p, kSPU); w.valid() && ok; w.next(), ++n_seg) {
             const int dbuf = n_seg % kDBufs;
             // the epilogue of the segment that used this accumulator before must have drained it
             if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
@@ -353,11 +370,13 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(stage0 + (size_t)r.slot * kStageBytes));
-                    const uint32_t a_t = tmem_base + kTileAColBase + r.slot * 32;
+                    const uint32_t a_t = tmem_base + kACol + r.slot * kSlotCols;
 #pragma unroll
-                    for (int kk = 0; kk < kTileStageK / 16; ++kk) {
-                        // 16 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled rows of B
-                        tc_mma_ts(d_t, a_t + kk * 8, bdesc + (uint64_t)(kk * 2), kIdesc, (j == 0 && kk == 0) ? 0u : 1u);
+                    for (int kk = 0; kk < kStageK / 16; ++kk) {
+                        // 16 k per instruction: 8 TMEM columns of A; in B 32 bytes along the swizzled rows of
+                        // a 64-k box, the next box MT * 128 bytes further
+                        const uint64_t bd = bdesc + (uint64_t)((kk / 4) * (MT * 128 / 16) + (kk % 4) * 2);
+                        tc_mma_ts(d_t, a_t + kk * 8, bd, kIdesc, (j == 0 && kk == 0) ? 0u : 1u);
                     }
                     tc_commit(&retired[r.slot]);
                     if (j == nst - 1) tc_commit(&d_full[dbuf]);
@@ -382,26 +401,30 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 
         // this set's first stage inside a segment
         auto first_own = [&](const SegWalk& w) { return (int)(((uint32_t)set - w.n0) & 3u); };
-        // packed words of stage j of the load walker's segment (zeros past the matrix edge)
-        auto load_stage = [&](const SegWalk& w, int j, StageRegs& r) {
+        // packed words of stage j of the load walker's segment (zeros past the matrix edge); a stage is
+        // a whole group (kSPU == 1) or one 64-k half of it
+        auto load_stage = [&](const SegWalk& w, int j, StageRegs<kNW>& r) {
             const int t64 = 2 * w.nt + half;                      // 64-column packed tile
             if (t64 * kTileN < p.N) {
-                const size_t blk = (size_t)t64 * p.G + (w.g0 + (j >> 1));
-                const uint32_t* wp = p.Wq + blk * kBlockWords + (j & 1) * 512;
-                r.w0 = __ldg(reinterpret_cast<const uint4*>(wp + wo0));
-                r.w1 = __ldg(reinterpret_cast<const uint4*>(wp + wo1));
+                const size_t blk = (size_t)t64 * p.G + (w.g0 + j / kSPU);
+                const uint32_t* wp = p.Wq + blk * kBlockWords + (j % kSPU) * 512;
+#pragma unroll
+                for (int h = 0; h < kNW / 2; ++h) {
+                    r.w[2 * h] = __ldg(reinterpret_cast<const uint4*>(wp + h * 512 + wo0));
+                    r.w[2 * h + 1] = __ldg(reinterpret_cast<const uint4*>(wp + h * 512 + wo1));
+                }
                 r.s = __ldg(reinterpret_cast<const unsigned short*>(p.S) + blk * kSBlockHalves + col);
                 r.zw = __ldg(p.Z + blk * kZBlockWords + (col >> 3));
             } else {
-                r.w0 = make_uint4(0, 0, 0, 0);
-                r.w1 = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int i = 0; i < kNW; ++i) r.w[i] = make_uint4(0, 0, 0, 0);
                 r.s = 0;
                 r.zw = 0;
             }
         };
 
-        // load cursor: runs kTilePrefetch of this set's stages ahead of the compute loop
-        SegWalk wl(p);
+        // load cursor: runs kPF of this set's stages ahead of the compute loop
+        SegWalk wl(p, kSPU);
         int jl = wl.valid() ? first_own(wl) : 0;
         auto settle = [&]() {   // move the cursor to a segment that still has a stage of this set
             while (wl.valid() && jl >= wl.stages_in_seg()) {
@@ -410,9 +433,9 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             }
         };
         settle();
-        StageRegs pf[kTilePrefetch];
+        StageRegs<kNW> pf[kPF];
 #pragma unroll
-        for (int i = 0; i < kTilePrefetch; ++i) {
+        for (int i = 0; i < kPF; ++i) {
             if (wl.valid()) {
                 load_stage(wl, jl, pf[i]);
                 jl += kTileSets;
@@ -425,17 +448,17 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         uint32_t n_seg = 0, n_prev = 0;
         RingPos rp{0, 0u};
         bool ok = true;
-        for (SegWalk w(p); w.valid() && ok; w.next(), ++n_seg) {
+        for (SegWalk w(p, kSPU); w.valid() && ok; w.next(), ++n_seg) {
             const int nst = w.stages_in_seg();
             for (int j = first_own(w); j < nst; j += kTileSets) {
                 const uint32_t n = w.n0 + (uint32_t)j;
                 rp.advance((int)(n - n_prev), R);
                 n_prev = n;
-                const StageRegs cur = pf[0];
+                const StageRegs<kNW> cur = pf[0];
 #pragma unroll
-                for (int i = 0; i + 1 < kTilePrefetch; ++i) pf[i] = pf[i + 1];
+                for (int i = 0; i + 1 < kPF; ++i) pf[i] = pf[i + 1];
                 if (wl.valid()) {
-                    load_stage(wl, jl, pf[kTilePrefetch - 1]);
+                    load_stage(wl, jl, pf[kPF - 1]);
                     jl += kTileSets;
                     settle();
                 }
@@ -445,9 +468,10 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 // the MMAs that read this slot one ring turn ago must have retired
                 if (n >= (uint32_t)R && !mbar_wait(&retired[rp.slot], rp.ph ^ 1u)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_t = tmem_base + lane_addr + kTileAColBase + rp.slot * 32;
-                {
-                    const uint32_t ww[4] = {cur.w0.x, cur.w0.y, cur.w0.z, cur.w0.w};   // k = 0 .. 31
+                const uint32_t a_t = tmem_base + lane_addr + kACol + rp.slot * kSlotCols;
+#pragma unroll
+                for (int c = 0; c < kNW; ++c) {      // 32 k -> 16 TMEM columns at a time
+                    const uint32_t ww[4] = {cur.w[c].x, cur.w[c].y, cur.w[c].z, cur.w[c].w};
                     uint32_t regs[16];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
@@ -455,18 +479,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll
                         for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
                     }
-                    tc_st16(a_t, regs);
-                }
-                {
-                    const uint32_t ww[4] = {cur.w1.x, cur.w1.y, cur.w1.z, cur.w1.w};   // k = 32 .. 63
-                    uint32_t regs[16];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
-                    }
-                    tc_st16(a_t + 16, regs);
+                    tc_st16(a_t + 16 * c, regs);
                 }
                 tc_wait_st();
                 tc_fence_before();
