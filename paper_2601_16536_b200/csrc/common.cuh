@@ -73,31 +73,42 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait: returns false (after recording the status code) if the phase never completes.
-// The whole poll loop is one asm block (a predicate branch straight off try_wait; about 40 clocks
-// when the phase is already complete).  try_wait itself blocks for a hardware-defined slice, so
-// the limit below is far beyond any legitimate wait, yet finite.
+// Bounded wait: returns false (after recording the status code) if the phase does not complete
+// within about two seconds.  Fast path: one try_wait (about 40 clocks when the phase is already
+// complete).  Slow path: try_wait with a suspend-time hint, so that a waiting warp sleeps in the
+// barrier unit instead of spending issue slots on polling, and a wall-clock limit read from
+// %globaltimer (the hint is only a hint: an iteration count would not bound the time).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t"
-        ".reg .pred p, q;\n\t"
-        ".reg .u32 cnt;\n\t"
-        "mov.u32 cnt, 0;\n\t"
-        "W4A16_WAIT_LOOP:\n\t"
+        ".reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "@p bra W4A16_WAIT_DONE;\n\t"
-        "add.u32 cnt, cnt, 1;\n\t"
-        "setp.lt.u32 q, cnt, 0x400000;\n\t"
-        "@q bra W4A16_WAIT_LOOP;\n\t"
-        "W4A16_WAIT_DONE:\n\t"
         "selp.u32 %0, 1, 0, p;\n\t"
         "}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
-    if (ok == 0) report_status(kStatusMbarTimeout);
-    return ok != 0;
+    if (ok) return true;
+    unsigned long long t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (;;) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
+            : "memory");
+        if (ok) return true;
+        unsigned long long t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        if (t1 - t0 > 2000000000ull) break;
+    }
+    report_status(kStatusMbarTimeout);
+    return false;
 }
 
 // One lane of a converged warp (warp-uniform control flow keeps addresses and descriptors in
