@@ -145,6 +145,17 @@ TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     g.tiles = (long)g.m_tiles * g.n_tiles;
     // more tiles than ticket counters: whole tiles only (no partial tiles, no tickets)
     if (split_k == 0 && g.tiles > kTileMaxTicketTiles) split_k = 1;
+    if (split_k == 0 && g.tiles <= sms) {
+        // Fewer tiles than SMs.  Balanced chunks use every SM, but a chunk that crosses a tile boundary
+        // drains an accumulator and goes through the ticket exchange in mid-stream, which stalls its
+        // pipeline for about as long as six groups take.  S slices per tile keep every chunk inside one
+        // tile at the price of idle SMs.  Take the cheaper of the two (cost in groups per CTA).
+        int s0 = sms / (int)g.tiles;
+        if (s0 > G) s0 = G;
+        const long classic_cost = (G + s0 - 1) / s0;
+        const long balanced_cost = (g.tiles * G + sms - 1) / sms + 6;
+        if (classic_cost <= balanced_cost) split_k = s0;
+    }
     g.split_k = split_k;
     if (split_k == 0) {
         const long units = g.tiles * G;
@@ -176,7 +187,7 @@ size_t tile_workspace_bytes(const TileGeom& g) {
 // Nominal split factor of the tile path's schedule: how many chunks share one tile's K range.
 int choose_split_tile(int M, int N, int G, int sms) {
     TileGeom g = tile_geom(M, N, G, 0, sms, 227 * 1024);
-    if (g.split_k == 1) return 1;
+    if (g.split_k >= 1) return g.split_k;
     long s = (g.nchunks + g.tiles - 1) / g.tiles;
     if (s < 1) s = 1;
     if (s > G) s = G;
