@@ -34,8 +34,9 @@
 // owns TMEM lanes 32 (w % 4) .. + 31.  Each thread keeps the packed words of its next few stages in
 // registers (loads issued that far ahead).  With MT <= 128 two accumulators alternate between
 // segments, so one drains while the next fills.  The packed weights do not depend on the previous
-// kernel in the stream: under programmatic dependent launch the first weight loads are issued
-// before griddepcontrol.wait, and only activations, C and the workspace are touched after it.
+// kernel in the stream: under programmatic dependent launch the dequant warps load and convert
+// weights until the TMEM ring is full before anything waits for that kernel; only activations, C
+// and the workspace are touched after griddepcontrol.wait.
 // The producer and MMA warps run warp-uniform loops and elect one lane per instruction, which
 // keeps descriptors in uniform registers.  All waits are bounded mbarrier waits; a wait that runs
 // out records a status code and the CTA drains and exits (TMEM is always released).
@@ -442,8 +443,10 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 settle();
             }
         }
-        // everything below may read or write memory the previous kernel is still writing
-        asm volatile("griddepcontrol.wait;" ::: "memory");
+        // Converting weights into the TMEM ring touches nothing the previous kernel may still be writing,
+        // so it starts at once and runs until the ring is full; the dependency wait comes before this
+        // warp's first write to global memory (the first epilogue).
+        bool dep_waited = false;
 
         uint32_t n_seg = 0, n_prev = 0;
         RingPos rp{0, 0u};
@@ -492,6 +495,10 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             const int dbuf = n_seg % kDBufs;
             if (!mbar_wait(&d_full[dbuf], (n_seg / kDBufs) & 1u)) { ok = false; break; }
             tc_fence_after();
+            if (!dep_waited) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                dep_waited = true;
+            }
             const int T = w.t;
             const int n = w.nt * kTileCols + row;
             const int m_base = w.mt_i * MT + set * kCW;     // first batch row of this warp's columns
