@@ -402,88 +402,106 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 
         // this set's first stage inside a segment
         auto first_own = [&](const SegWalk& w) { return (int)(((uint32_t)set - w.n0) & 3u); };
-        // packed words of stage j of the load walker's segment (zeros past the matrix edge); a stage is
-        // a whole group (kSPU == 1) or one 64-k half of it
-        auto load_stage = [&](const SegWalk& w, int j, StageRegs<kNW>& r) {
-            const int t64 = 2 * w.nt + half;                      // 64-column packed tile
-            if (t64 * kTileN < p.N) {
-                const size_t blk = (size_t)t64 * p.G + (w.g0 + j / kSPU);
-                const uint32_t* wp = p.Wq + blk * kBlockWords + (j % kSPU) * 512;
+        // Load cursor: runs kPF of this set's stages ahead of the compute loop.  Inside a segment this
+        // set's stages are kTileSets apart (kTileSets / kSPU groups on, same part of the group), so the
+        // three pointers just step; they are recomputed only when the cursor enters a new segment.
+        SegWalk wl(p, kSPU);
+        int jl = 0;
+        bool l_in = false;                      // this thread's column exists (not past the matrix edge)
+        const uint32_t* lw = nullptr;           // the stage's first word of this thread's 8-column block
+        const unsigned short* ls = nullptr;
+        const uint32_t* lz = nullptr;
+        auto point = [&]() {                    // cursor entered a new segment: settle on a stage, set pointers
+            while (wl.valid()) {
+                jl = first_own(wl);
+                if (jl < wl.stages_in_seg()) break;
+                wl.next();
+            }
+            if (!wl.valid()) return;
+            const int t64 = 2 * wl.nt + half;   // 64-column packed tile
+            l_in = t64 * kTileN < p.N;
+            const size_t blk = (size_t)t64 * p.G + (wl.g0 + jl / kSPU);
+            lw = p.Wq + blk * kBlockWords + (jl % kSPU) * 512;
+            ls = reinterpret_cast<const unsigned short*>(p.S) + blk * kSBlockHalves + col;
+            lz = p.Z + blk * kZBlockWords + (col >> 3);
+        };
+        // load the cursor's stage (zeros past the matrix edge) and advance the cursor
+        auto fetch = [&](StageRegs<kNW>& r) {
+            if (!wl.valid()) return;
+            if (l_in) {
 #pragma unroll
                 for (int h = 0; h < kNW / 2; ++h) {
-                    r.w[2 * h] = __ldg(reinterpret_cast<const uint4*>(wp + h * 512 + wo0));
-                    r.w[2 * h + 1] = __ldg(reinterpret_cast<const uint4*>(wp + h * 512 + wo1));
+                    r.w[2 * h] = __ldg(reinterpret_cast<const uint4*>(lw + h * 512 + wo0));
+                    r.w[2 * h + 1] = __ldg(reinterpret_cast<const uint4*>(lw + h * 512 + wo1));
                 }
-                r.s = __ldg(reinterpret_cast<const unsigned short*>(p.S) + blk * kSBlockHalves + col);
-                r.zw = __ldg(p.Z + blk * kZBlockWords + (col >> 3));
+                r.s = __ldg(ls);
+                r.zw = __ldg(lz);
             } else {
 #pragma unroll
                 for (int i = 0; i < kNW; ++i) r.w[i] = make_uint4(0, 0, 0, 0);
                 r.s = 0;
                 r.zw = 0;
             }
-        };
-
-        // load cursor: runs kPF of this set's stages ahead of the compute loop
-        SegWalk wl(p, kSPU);
-        int jl = wl.valid() ? first_own(wl) : 0;
-        auto settle = [&]() {   // move the cursor to a segment that still has a stage of this set
-            while (wl.valid() && jl >= wl.stages_in_seg()) {
+            jl += kTileSets;
+            if (jl < wl.stages_in_seg()) {
+                lw += (kTileSets / kSPU) * kBlockWords;
+                ls += (kTileSets / kSPU) * kSBlockHalves;
+                lz += (kTileSets / kSPU) * kZBlockWords;
+            } else {
                 wl.next();
-                if (wl.valid()) jl = first_own(wl);
+                point();
             }
         };
-        settle();
-        StageRegs<kNW> pf[kPF];
-#pragma unroll
-        for (int i = 0; i < kPF; ++i) {
-            if (wl.valid()) {
-                load_stage(wl, jl, pf[i]);
-                jl += kTileSets;
-                settle();
-            }
-        }
+        point();
+        // register ring of prefetched stages, written out so that no slot is ever copied
+        static_assert(kPF == 2 || kPF == 3, "the ring below has two or three slots");
+        StageRegs<kNW> pf0, pf1, pf2;
+        fetch(pf0);
+        fetch(pf1);
+        if (kPF == 3) fetch(pf2);
         // Converting weights into the TMEM ring touches nothing the previous kernel may still be writing,
         // so it starts at once and runs until the ring is full; the dependency wait comes before this
         // warp's first write to global memory (the first epilogue).
         bool dep_waited = false;
 
         uint32_t n_seg = 0, n_prev = 0;
+        int pi = 0;                             // ring slot that holds the next stage to convert
         RingPos rp{0, 0u};
         bool ok = true;
+        // one stage of this thread's column -> kSlotCols TMEM columns of the ring slot
+        auto convert = [&](const StageRegs<kNW>& cur, uint32_t n) -> bool {
+            const uint32_t z = (cur.zw >> zsh) & 15u;
+            const __half2 s2 = u32_as_h2(cur.s * 0x00010001u);
+            const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
+            // the MMAs that read this slot one ring turn ago must have retired
+            if (n >= (uint32_t)R && !mbar_wait(&retired[rp.slot], rp.ph ^ 1u)) return false;
+            tc_fence_after();
+            const uint32_t a_t = tmem_base + lane_addr + kACol + rp.slot * kSlotCols;
+#pragma unroll
+            for (int c = 0; c < kNW; ++c) {      // 32 k -> 16 TMEM columns at a time
+                const uint32_t ww[4] = {cur.w[c].x, cur.w[c].y, cur.w[c].z, cur.w[c].w};
+                uint32_t regs[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
+                }
+                tc_st16(a_t + 16 * c, regs);
+            }
+            return true;
+        };
         for (SegWalk w(p, kSPU); w.valid() && ok; w.next(), ++n_seg) {
             const int nst = w.stages_in_seg();
             for (int j = first_own(w); j < nst; j += kTileSets) {
                 const uint32_t n = w.n0 + (uint32_t)j;
                 rp.advance((int)(n - n_prev), R);
                 n_prev = n;
-                const StageRegs<kNW> cur = pf[0];
-#pragma unroll
-                for (int i = 0; i + 1 < kPF; ++i) pf[i] = pf[i + 1];
-                if (wl.valid()) {
-                    load_stage(wl, jl, pf[kPF - 1]);
-                    jl += kTileSets;
-                    settle();
-                }
-                const uint32_t z = (cur.zw >> zsh) & 15u;
-                const __half2 s2 = u32_as_h2(cur.s * 0x00010001u);
-                const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
-                // the MMAs that read this slot one ring turn ago must have retired
-                if (n >= (uint32_t)R && !mbar_wait(&retired[rp.slot], rp.ph ^ 1u)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t a_t = tmem_base + lane_addr + kACol + rp.slot * kSlotCols;
-#pragma unroll
-                for (int c = 0; c < kNW; ++c) {      // 32 k -> 16 TMEM columns at a time
-                    const uint32_t ww[4] = {cur.w[c].x, cur.w[c].y, cur.w[c].z, cur.w[c].w};
-                    uint32_t regs[16];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
-                    }
-                    tc_st16(a_t + 16 * c, regs);
-                }
+                // convert ring slot pi, then refill it with the stage kPF ahead
+                if (pi == 0) { ok = convert(pf0, n); fetch(pf0); pi = 1; }
+                else if (pi == 1) { ok = convert(pf1, n); fetch(pf1); pi = (kPF == 3) ? 2 : 0; }
+                else { ok = convert(pf2, n); fetch(pf2); pi = 0; }
+                if (!ok) break;
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
