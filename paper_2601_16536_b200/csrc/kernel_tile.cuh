@@ -555,8 +555,9 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 // Split-K reduce (Algorithm 1, Phase 3), per warp region (32 columns n x MT/4 rows m)
                 __threadfence();
                 __syncwarp();
-                const int c_first = tile_chunk_of(p, tile_u0);
-                const int c_last = tile_chunk_of(p, tile_u0 + p.G - 1);
+                // (classic slices: no division on the way to the ticket)
+                const int c_first = p.split_k > 0 ? T * p.split_k : tile_chunk_of(p, tile_u0);
+                const int c_last = p.split_k > 0 ? c_first + p.split_k - 1 : tile_chunk_of(p, tile_u0 + p.G - 1);
                 int* ticket = p.tickets + ((size_t)T * kTileDequantWarps + dw);
                 int last = 0;
                 if (lane == 0) {
@@ -572,7 +573,8 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                     // summed kStep at a time so that many loads are in flight.
                     const size_t slot_elems = (size_t)MT * kTileCols;
                     const float* base = p.ws + (size_t)(set * kCW) * kTileCols + row;
-                    const size_t first_slot = 2 * (size_t)c_first + (tile_chunk_begin(p, c_first) == tile_u0 ? 0 : 1);
+                    const size_t first_slot =
+                        2 * (size_t)c_first + ((p.split_k > 0 || tile_chunk_begin(p, c_first) == tile_u0) ? 0 : 1);
 #pragma unroll 1
                     for (int m0 = 0; m0 < kCW; m0 += kStep) {
                         float acc[kStep];
