@@ -145,15 +145,24 @@ TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     g.tiles = (long)g.m_tiles * g.n_tiles;
     // more tiles than ticket counters: whole tiles only (no partial tiles, no tickets)
     if (split_k == 0 && g.tiles > kTileMaxTicketTiles) split_k = 1;
-    if (split_k == 0 && g.tiles <= sms) {
-        // Fewer tiles than SMs.  Balanced chunks use every SM, but a chunk that crosses a tile boundary
-        // drains an accumulator and goes through the ticket exchange in mid-stream, which stalls its
-        // pipeline for about as long as six groups take.  S slices per tile keep every chunk inside one
-        // tile at the price of idle SMs.  Take the cheaper of the two (cost in groups per CTA).
-        int s0 = sms / (int)g.tiles;
-        if (s0 > G) s0 = G;
-        const long classic_cost = (G + s0 - 1) / s0;
-        const long balanced_cost = (g.tiles * G + sms - 1) / sms + 6;
+    if (split_k == 0) {
+        // Balanced chunks use every SM to the end, but a chunk that starts or ends inside a tile leaves
+        // an FP32 partial tile behind (store, ticket, reload: the larger the batch tile the dearer, and
+        // in mid-stream it stalls the pipeline).  S slices per tile (tiles <= SMs) or whole tiles in
+        // waves (tiles > SMs) avoid that at the price of idle SMs.  Cost model in groups per CTA; the
+        // constants are fitted to measurements (K = 11008 / N = 4096, K = 28672 / N = 8192 and
+        // K = N = 8192 with M up to 4096).
+        const long penalty = 6 + g.mt / 8;
+        const long balanced_cost = (g.tiles * G + sms - 1) / sms + penalty;
+        int s0 = 1;
+        long classic_cost;
+        if (g.tiles <= sms) {
+            s0 = sms / (int)g.tiles;
+            if (s0 > G) s0 = G;
+            classic_cost = (G + s0 - 1) / s0;
+        } else {
+            classic_cost = ((g.tiles + sms - 1) / sms) * G;
+        }
         if (classic_cost <= balanced_cost) split_k = s0;
     }
     g.split_k = split_k;
