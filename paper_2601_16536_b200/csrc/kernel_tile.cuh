@@ -28,18 +28,26 @@
 // No warp ever waits for another CTA, and the order of the sum is fixed, so results are
 // bit-identical from run to run.
 //
-// One pipeline stage is 64 k.  A ring of R <= 8 slots holds, per slot, the MT x 64 FP16 activation
-// box in shared memory and 32 TMEM columns of dequantized weights; the MMAs of a stage release both
-// with one commit.  Four sets of four dequant warps take stages round-robin; inside a set warp w
-// owns TMEM lanes 32 (w % 4) .. + 31.  Each thread keeps the packed words of its next few stages in
-// registers (loads issued that far ahead).  With MT <= 128 two accumulators alternate between
-// segments, so one drains while the next fills.  The packed weights do not depend on the previous
-// kernel in the stream: under programmatic dependent launch the dequant warps load and convert
-// weights until the TMEM ring is full before anything waits for that kernel; only activations, C
-// and the workspace are touched after griddepcontrol.wait.
+// One pipeline stage is a whole group (128 k, eight MMAs) for batch tiles of up to 64 rows and half
+// a group (64 k, four MMAs) above: narrow tiles are bound by the per-stage hand-offs and by the
+// issuing lane (about 40 clocks per tcgen05.mma whatever its size), wide ones by the tensor pipe.
+// A ring of R slots holds, per slot, the stage's activation boxes in shared memory and its
+// dequantized weights in tensor memory (32 or 64 columns; six or eight slots fit beside the
+// accumulators); the MMAs of a stage release both with one commit.  Four sets of four dequant
+// warps take stages round-robin; inside a set warp w owns TMEM lanes 32 (w % 4) .. + 31.  Each
+// thread keeps the packed words of its next two or three stages in registers (loads issued that
+// far ahead, pointers stepped, no register copies).  With MT <= 128 two accumulators alternate
+// between segments, so one drains while the next fills.  The packed weights do not depend on the
+// previous kernel in the stream: under programmatic dependent launch the dequant warps load and
+// convert weights until the TMEM ring is full before anything waits for that kernel; only
+// activations, C and the workspace are touched after griddepcontrol.wait.
 // The producer and MMA warps run warp-uniform loops and elect one lane per instruction, which
 // keeps descriptors in uniform registers.  All waits are bounded mbarrier waits; a wait that runs
 // out records a status code and the CTA drains and exits (TMEM is always released).
+//
+// Which schedule a shape gets when the caller leaves split_k open is the host's choice (api.cu):
+// partial tiles are dear (FP32 store, ticket, reload; in mid-chunk they also stall the pipeline), so
+// balanced chunks are used only where the SMs left idle by whole slices or whole tiles cost more.
 #pragma once
 
 #include <cuda.h>
