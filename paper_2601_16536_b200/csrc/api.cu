@@ -241,11 +241,21 @@ EncodeTiledFn encode_tiled_fn() {
 bool make_act_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mt) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTileBoxK, (cuuint32_t)mt};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(A), dims, strides, box, estr,
+    if (tile_stage_k(mt) == kTileBoxK) {     // one box per stage: plain 2-D tensor, k innermost
+        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+        const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kTileBoxK, (cuuint32_t)mt};
+        const cuuint32_t estr[2] = {1, 1};
+        return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(A), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
+    // A[M][K] seen as [K / 64][M][64]: one copy brings a stage's 64-k boxes one after the other
+    const cuuint64_t dims[3] = {(cuuint64_t)kTileBoxK, (cuuint64_t)M, (cuuint64_t)(K / kTileBoxK)};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)kTileBoxK * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kTileBoxK, (cuuint32_t)mt, (cuuint32_t)(tile_stage_k(mt) / kTileBoxK)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(A), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -478,7 +488,7 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
         // tail of the previous kernel in the stream; it orders itself with griddepcontrol.wait
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(g.ctas, 1, 1);
-        cfg.blockDim = dim3(kTileThreads, 1, 1);
+        cfg.blockDim = dim3(tile_threads(g.mt), 1, 1);
         cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];

@@ -63,7 +63,16 @@ constexpr int kTileBoxK = 64;                       // k per activation TMA box 
 __host__ __device__ constexpr int tile_stage_k(int mt) { return mt <= 64 ? 128 : 64; }
 constexpr int kTileDequantWarps = 16;               // four sets of four (one warp per TMEM lane quarter)
 constexpr int kTileSets = kTileDequantWarps / 4;
-constexpr int kTileThreads = (2 + kTileDequantWarps) * 32;   // producer, MMA, dequant/epilogue warps
+// MMA-issuing warps.  A narrow batch tile is bound by the issuing warp's own loop (a lone warp of
+// dependent scalar code next to sixteen busy dequant warps gets through a stage in 600 to 700 clocks,
+// of which the eight MMAs are about 100), so there the stages are dealt to several issuers, each with
+// an accumulator of its own; the epilogue adds the accumulators in issuer order.
+__host__ __device__ constexpr int tile_issuers(int mt) { return mt <= 32 ? 3 : mt <= 64 ? 2 : 1; }
+// producer, issuers, dequant / epilogue warps
+__host__ __device__ constexpr int tile_threads(int mt) { return (1 + tile_issuers(mt) + kTileDequantWarps) * 32; }
+// accumulators per issuer that alternate between segments, and the TMEM columns between accumulators
+__host__ __device__ constexpr int tile_dbufs(int mt) { return mt <= 16 ? 2 : mt <= 64 ? 1 : mt <= 128 ? 2 : 1; }
+__host__ __device__ constexpr int tile_d_stride(int mt) { return mt <= 64 ? mt : 128; }
 constexpr int kTileMaxStages = 8;                   // ring slots: activation boxes + stage_k / 2 TMEM columns each
 // TMEM columns: the accumulators first (two of up to 128 columns, or one of 256), then the operand ring
 __host__ __device__ constexpr int tile_a_col_base(int mt) { return mt <= 64 ? 128 : 256; }
@@ -94,6 +103,12 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
         : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -257,15 +272,32 @@ struct SegWalk {
     __device__ __forceinline__ bool whole_tile() const { return g0 == 0 && units == p.G; }
 };
 
-// Position in the ring of R slots: slot = n % R, phase = (n / R) & 1, kept incrementally.
+// Position in the ring of R slots: slot = n % R, turn = n / R, phase = turn & 1, kept incrementally.
 struct RingPos {
     int slot;
     uint32_t ph;
+    uint32_t turn;
     __device__ __forceinline__ void advance(int d, int R) {
         slot += d;
-        while (slot >= R) { slot -= R; ph ^= 1u; }
+        while (slot >= R) { slot -= R; ph ^= 1u; ++turn; }
     }
 };
+
+// "The MMAs that read this slot have retired" has TWO barriers per slot, used by alternate ring turns.
+// A parity wait tells a phase from the one before it, not from the one two back, so whoever waits on
+// a barrier must see every one of its phases.  The producer does (it walks every stage).  A dequant
+// set takes every fourth stage, and with six slots it comes back to a slot only every second turn;
+// with one barrier per slot it would skip a phase each time, and nothing but a single in-order issuer
+// would keep the skipped phase from still being open.  With one barrier per slot and turn parity the
+// set meets the same barrier on every visit and that barrier completes exactly one phase in between.
+__device__ __forceinline__ uint64_t* retired_bar(uint64_t* retired, const RingPos& r) {
+    return retired + (r.turn & 1u) * kTileMaxStages + r.slot;      // the stage at r commits here
+}
+// until the stage that used r's slot one ring turn earlier has retired (r.turn >= 1)
+__device__ __forceinline__ bool wait_slot_free(uint64_t* retired, const RingPos& r) {
+    const uint32_t t = r.turn - 1u;
+    return mbar_wait(retired + (t & 1u) * kTileMaxStages + r.slot, (t >> 1) & 1u);
+}
 
 // Packed words, scale and zero point of one thread's column for one stage of 32 * NW k.
 template <int NW>
@@ -276,7 +308,7 @@ struct StageRegs {
 };
 
 template <int MT>
-__global__ void __launch_bounds__(kTileThreads, 1)
+__global__ void __launch_bounds__(tile_threads(MT), 1)
 gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // 1024-byte alignment of the stage buffers (the swizzle atom) regardless of where the
@@ -285,8 +317,9 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     constexpr int kStageBytes = tile_stage_bytes(MT);
     constexpr uint32_t kIdesc = tile_idesc(MT);
     constexpr int kCW = MT / kTileSets;                  // accumulator columns (batch rows) per epilogue warp
-    constexpr int kDBufs = MT <= 128 ? 2 : 1;            // accumulators in TMEM
-    constexpr int kDStride = MT <= 64 ? 64 : 128;        // column distance between the two
+    constexpr int kNI = tile_issuers(MT);                // MMA-issuing warps, one accumulator (set) each
+    constexpr int kDBufs = tile_dbufs(MT);               // accumulators per issuer: accumulator (b, i) sits
+    constexpr int kDStride = tile_d_stride(MT);          // at column (b * kNI + i) * kDStride
     constexpr int kStageK = tile_stage_k(MT);            // k per ring slot
     constexpr int kSPU = kGroup / kStageK;               // stages per unit
     constexpr int kSlotCols = kStageK / 2;               // TMEM columns of one operand slot
@@ -295,8 +328,8 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     constexpr int kPF = tile_prefetch(MT);
 
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [R]  activation box landed AND operand stored in TMEM
-    uint64_t* retired = full + kTileMaxStages;                   // [R]  the stage's MMAs retired: slot free
-    uint64_t* d_full = retired + kTileMaxStages;                 // [2]  accumulator complete
+    uint64_t* retired = full + kTileMaxStages;                   // [2][R]  the stage's MMAs retired: slot free
+    uint64_t* d_full = retired + 2 * kTileMaxStages;             // [2]  accumulator complete
     uint64_t* d_empty = d_full + 2;                              // [2]  accumulator drained by the epilogue
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(d_empty + 2);
     int* flags = reinterpret_cast<int*>(tmem_slot + 1);          // [0] a bounded wait ran out, [1] stages issued
@@ -309,9 +342,10 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         for (int i = 0; i < R; ++i) {
             mbar_init(&full[i], 1 + 4);      // the producer's arrive.expect_tx + one arrival per warp of a dequant set
             mbar_init(&retired[i], 1);
+            mbar_init(&retired[kTileMaxStages + i], 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&d_full[i], 1);
+            mbar_init(&d_full[i], kNI);      // every issuer reports once per segment
             mbar_init(&d_empty[i], kTileDequantWarps);
         }
         flags[0] = 0;
@@ -337,23 +371,24 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         if (elect_one()) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         asm volatile("griddepcontrol.wait;" ::: "memory");   // activations may come from the previous kernel
         bool ok = true;
-        RingPos r{0, 0u};
+        RingPos r{0, 0u, 0u};
         uint32_t n = 0;
         for (SegWalk w(p, kSPU); w.valid() && ok; w.next()) {
-            int k = w.g0 * kGroup;
+            int kb = w.g0 * (kGroup / kTileBoxK);            // 64-k box index along K
             const int m = w.mt_i * MT;
             const int nst = w.stages_in_seg();
             for (int j = 0; j < nst; ++j) {
-                if (n >= (uint32_t)R && !mbar_wait(&retired[r.slot], r.ph ^ 1u)) { ok = false; break; }
+                if (r.turn != 0u && !wait_slot_free(retired, r)) { ok = false; break; }
                 if (elect_one()) {
+                    // one copy per stage: kStageK / 64 boxes of MT rows x 64 k, box b at b * MT * 128 bytes
                     mbar_expect_tx(&full[r.slot], (uint32_t)kStageBytes);
-#pragma unroll
-                    for (int b = 0; b < kStageK / kTileBoxK; ++b)
-                        tma_load_2d(stage0 + (size_t)r.slot * kStageBytes + b * (MT * 128), &tmap_a, k + b * kTileBoxK, m,
-                                    &full[r.slot]);
+                    if constexpr (kStageK == kTileBoxK)
+                        tma_load_2d(stage0 + (size_t)r.slot * kStageBytes, &tmap_a, kb * kTileBoxK, m, &full[r.slot]);
+                    else
+                        tma_load_3d(stage0 + (size_t)r.slot * kStageBytes, &tmap_a, 0, m, kb, &full[r.slot]);
                 }
                 __syncwarp();
-                k += kStageK;
+                kb += kStageK / kTileBoxK;
                 ++n;
                 r.advance(1, R);
             }
@@ -362,19 +397,33 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             flags[1] = (int)n;
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp <= kNI) {
+        // ------------------------------------------------------------ MMA issuer `iss`: the stages whose
+        // index in this CTA is = iss (mod kNI), summed into this issuer's own accumulator
+        const int iss = warp - 1;
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        uint32_t n_seg = 0;
+        uint32_t n_seg = 0, n_prev = 0;
         bool ok = true;
-        RingPos r{0, 0u};
+        RingPos r{0, 0u, 0u};
         for (SegWalk w(p, kSPU); w.valid() && ok; w.next(), ++n_seg) {
             const int dbuf = n_seg % kDBufs;
-            // the epilogue of the segment that used this accumulator before must have drained it
+            // the epilogue of the segment that used this accumulator before must have drained it (an
+            // issuer without a stage in this segment waits too, so that its report below cannot land
+            // in the barrier phase of that earlier segment)
             if (!mbar_wait(&d_empty[dbuf], ((n_seg / kDBufs) & 1u) ^ 1u)) { ok = false; break; }
-            const uint32_t d_t = tmem_base + dbuf * kDStride;
+            const uint32_t d_t = tmem_base + (dbuf * kNI + iss) * kDStride;
             const int nst = w.stages_in_seg();
-            for (int j = 0; j < nst; ++j) {
+            int j = kNI == 1 ? 0 : (int)(((uint32_t)(iss + kNI) - w.n0 % kNI) % kNI);
+            if (j >= nst) {
+                if (elect_one()) mbar_arrive(&d_full[dbuf]);     // nothing of mine in this segment
+                __syncwarp();
+                continue;
+            }
+            uint32_t acc = 0u;                                   // the segment's first MMA overwrites
+            for (; j < nst; j += kNI) {
+                const uint32_t n = w.n0 + (uint32_t)j;
+                r.advance((int)(n - n_prev), R);
+                n_prev = n;
                 if (!mbar_wait(&full[r.slot], r.ph)) { ok = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
@@ -385,19 +434,19 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                         // 16 k per instruction: 8 TMEM columns of A; in B 32 bytes along the swizzled rows of
                         // a 64-k box, the next box MT * 128 bytes further
                         const uint64_t bd = bdesc + (uint64_t)((kk / 4) * (MT * 128 / 16) + (kk % 4) * 2);
-                        tc_mma_ts(d_t, a_t + kk * 8, bd, kIdesc, (j == 0 && kk == 0) ? 0u : 1u);
+                        tc_mma_ts(d_t, a_t + kk * 8, bd, kIdesc, kk == 0 ? acc : 1u);
                     }
-                    tc_commit(&retired[r.slot]);
-                    if (j == nst - 1) tc_commit(&d_full[dbuf]);
+                    tc_commit(retired_bar(retired, r));
+                    if (j + kNI >= nst) tc_commit(&d_full[dbuf]);
                 }
                 __syncwarp();
-                r.advance(1, R);
+                acc = 1u;
             }
         }
         if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------ dequant + epilogue warps
-        const int dw = warp - 2;               // 0..15
+        const int dw = warp - (1 + kNI);       // 0..15
         const int set = dw >> 2;               // takes the stages whose index in this CTA is = set (mod 4)
         const int quarter = warp & 3;          // TMEM lanes this warp may touch
         const int row = quarter * 32 + lane;   // column n inside the CTA tile = TMEM lane
@@ -474,7 +523,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 
         uint32_t n_seg = 0, n_prev = 0;
         int pi = 0;                             // ring slot that holds the next stage to convert
-        RingPos rp{0, 0u};
+        RingPos rp{0, 0u, 0u};
         bool ok = true;
         // one stage of this thread's column -> kSlotCols TMEM columns of the ring slot
         auto convert = [&](const StageRegs<kNW>& cur, uint32_t n) -> bool {
@@ -482,7 +531,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             const __half2 s2 = u32_as_h2(cur.s * 0x00010001u);
             const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
             // the MMAs that read this slot one ring turn ago must have retired
-            if (n >= (uint32_t)R && !mbar_wait(&retired[rp.slot], rp.ph ^ 1u)) return false;
+            if (rp.turn != 0u && !wait_slot_free(retired, rp)) return false;
             tc_fence_after();
             const uint32_t a_t = tmem_base + lane_addr + kACol + rp.slot * kSlotCols;
 #pragma unroll
@@ -528,7 +577,9 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             const int T = w.t;
             const int n = w.nt * kTileCols + row;
             const int m_base = w.mt_i * MT + set * kCW;     // first batch row of this warp's columns
-            const uint32_t d_t = tmem_base + lane_addr + dbuf * kDStride + set * kCW;
+            const uint32_t d_t = tmem_base + lane_addr + (dbuf * kNI) * kDStride + set * kCW;
+            // first stage of each issuer inside this segment: an issuer with none has no sum to add
+            const int iss0 = (int)(w.n0 % kNI);
             const long long tile_u0 = (long long)T * p.G;
             const bool whole = w.whole_tile();
             // first segment of a chunk -> slot 2 ci, its continuation into a later tile -> 2 ci + 1
@@ -537,10 +588,27 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll 1
             for (int cc = 0; cc < kCW; cc += kStep) {
                 uint32_t v[kStep];
-                if constexpr (kStep == 16) tc_ld16(d_t + cc, v);
-                else if constexpr (kStep == 8) tc_ld8(d_t + cc, v);
-                else tc_ld4(d_t + cc, v);
-                tc_wait_ld();
+                if constexpr (kNI == 1) {
+                    if constexpr (kStep == 16) tc_ld16(d_t + cc, v);
+                    else if constexpr (kStep == 8) tc_ld8(d_t + cc, v);
+                    else tc_ld4(d_t + cc, v);
+                    tc_wait_ld();
+                }
+                // several issuers: add their sums in stage order (issuer iss0 took the segment's first stage)
+#pragma unroll
+                for (int ii = 0; ii < (kNI == 1 ? 0 : kNI); ++ii) {
+                    if (ii >= nst) break;                        // warp-uniform
+                    int i = iss0 + ii;
+                    if (i >= kNI) i -= kNI;
+                    uint32_t t[kStep];
+                    if constexpr (kStep == 16) tc_ld16(d_t + i * kDStride + cc, t);
+                    else if constexpr (kStep == 8) tc_ld8(d_t + i * kDStride + cc, t);
+                    else tc_ld4(d_t + i * kDStride + cc, t);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int q = 0; q < kStep; ++q)
+                        v[q] = ii == 0 ? t[q] : __float_as_uint(__uint_as_float(v[q]) + __uint_as_float(t[q]));
+                }
                 if (whole) {
                     if (n < p.N) {
 #pragma unroll
