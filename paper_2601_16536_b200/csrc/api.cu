@@ -195,6 +195,10 @@ TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     int st = avail / tile_stage_bytes(g.mt);
     if (st > kTileMaxStages) st = kTileMaxStages;
     if (st > tile_max_slots(g.mt)) st = tile_max_slots(g.mt);   // the ring also lives in tensor memory
+    // parity waits tell a barrier phase only from its neighbour: every issuer has to come back to a slot
+    // on every ring turn and every dequant set on every turn or every second one (kernel_tile.cuh)
+    const int ring_unit = tile_issuers(g.mt) % 2 == 0 ? tile_issuers(g.mt) : 2 * tile_issuers(g.mt);
+    st -= st % ring_unit;                                        // 0 (no valid ring) is refused by the caller
     g.stages = st;
     g.smem_bytes = kTileBarBytes + 1024 + st * tile_stage_bytes(g.mt);
     // each CTA takes the SM's whole tensor memory: ask for enough shared memory that two never share an SM

@@ -63,15 +63,19 @@ constexpr int kTileBoxK = 64;                       // k per activation TMA box 
 __host__ __device__ constexpr int tile_stage_k(int mt) { return mt <= 64 ? 128 : 64; }
 constexpr int kTileDequantWarps = 16;               // four sets of four (one warp per TMEM lane quarter)
 constexpr int kTileSets = kTileDequantWarps / 4;
-// MMA-issuing warps.  A narrow batch tile is bound by the issuing warp's own loop (a lone warp of
-// dependent scalar code next to sixteen busy dequant warps gets through a stage in 600 to 700 clocks,
-// of which the eight MMAs are about 100), so there the stages are dealt to several issuers, each with
-// an accumulator of its own; the epilogue adds the accumulators in issuer order.
-__host__ __device__ constexpr int tile_issuers(int mt) { return mt <= 32 ? 3 : mt <= 64 ? 2 : 1; }
+// MMA-issuing warps.  With narrow batch tiles one issuing warp is busy nearly all the time (a lone
+// warp of dependent scalar code beside sixteen busy dequant warps needs 600 to 700 clocks per stage,
+// of which the eight MMAs are about 100), so for tiles of up to 32 rows the stages are dealt to three
+// issuers, each with an accumulator of its own; the epilogue adds the accumulators in issuer order.
+// Measured at K = 11008, N = 4096: 14.0 -> 13.0 us at M = 16; 64-row tiles are faster with one issuer
+// and two alternating accumulators (16.9 against 18.3 us), so the split stops at 32 rows.
+// An issuer must meet every phase of the `full` barriers it waits on, and a dequant set every phase
+// of its `retired` barriers: the ring size has to be an even multiple of the issuer count (host).
+__host__ __device__ constexpr int tile_issuers(int mt) { return mt <= 32 ? 3 : 1; }
 // producer, issuers, dequant / epilogue warps
 __host__ __device__ constexpr int tile_threads(int mt) { return (1 + tile_issuers(mt) + kTileDequantWarps) * 32; }
 // accumulators per issuer that alternate between segments, and the TMEM columns between accumulators
-__host__ __device__ constexpr int tile_dbufs(int mt) { return mt <= 16 ? 2 : mt <= 64 ? 1 : mt <= 128 ? 2 : 1; }
+__host__ __device__ constexpr int tile_dbufs(int mt) { return mt <= 16 ? 2 : mt <= 32 ? 1 : mt <= 128 ? 2 : 1; }
 __host__ __device__ constexpr int tile_d_stride(int mt) { return mt <= 64 ? mt : 128; }
 constexpr int kTileMaxStages = 8;                   // ring slots: activation boxes + stage_k / 2 TMEM columns each
 // TMEM columns: the accumulators first (two of up to 128 columns, or one of 256), then the operand ring
