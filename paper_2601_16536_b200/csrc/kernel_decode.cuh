@@ -352,8 +352,22 @@ __global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodePa
                     for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
                         const int n = idx & (kTileN - 1), m = idx >> 6;
                         float v = __ldcg(ws_mz + (size_t)first_slot * (kRows * kTileN) + idx);
-                        for (int c = c_first + 1; c <= c_last; ++c)
-                            v += __ldcg(ws_mz + (size_t)(2 * c) * (kRows * kTileN) + idx);
+                        // four loads in flight at a time (a load per round trip would make the tail
+                        // S - 1 trips long); the additions keep the ascending order
+                        const float* src = ws_mz + idx;
+                        const size_t cstride = (size_t)2 * (kRows * kTileN);
+                        int c = c_first + 1;
+                        for (; c + 3 <= c_last; c += 4) {
+                            const float x0 = __ldcg(src + (size_t)c * cstride), x1 = __ldcg(src + (size_t)(c + 1) * cstride);
+                            const float x2 = __ldcg(src + (size_t)(c + 2) * cstride), x3 = __ldcg(src + (size_t)(c + 3) * cstride);
+                            v += x0; v += x1; v += x2; v += x3;
+                        }
+                        if (c + 1 <= c_last) {
+                            const float x0 = __ldcg(src + (size_t)c * cstride), x1 = __ldcg(src + (size_t)(c + 1) * cstride);
+                            v += x0; v += x1;
+                            c += 2;
+                        }
+                        if (c <= c_last) v += __ldcg(src + (size_t)c * cstride);
                         p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
                     }
                 }

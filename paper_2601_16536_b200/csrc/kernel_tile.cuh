@@ -661,7 +661,21 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll
                         for (int q = 0; q < kStep; ++q)
                             acc[q] = __ldcg(base + first_slot * slot_elems + (size_t)(m0 + q) * kTileCols);
-                        for (int c = c_first + 1; c <= c_last; ++c) {
+                        // two contributors' loads in flight at a time (one per round trip would make
+                        // the tail S - 1 trips long); the additions keep the ascending order
+                        int c = c_first + 1;
+                        for (; c + 1 <= c_last; c += 2) {
+                            const float* src = base + (size_t)(2 * c) * slot_elems + (size_t)m0 * kTileCols;
+                            float x0[kStep], x1[kStep];
+#pragma unroll
+                            for (int q = 0; q < kStep; ++q) {
+                                x0[q] = __ldcg(src + (size_t)q * kTileCols);
+                                x1[q] = __ldcg(src + 2 * slot_elems + (size_t)q * kTileCols);
+                            }
+#pragma unroll
+                            for (int q = 0; q < kStep; ++q) { acc[q] += x0[q]; acc[q] += x1[q]; }
+                        }
+                        if (c <= c_last) {
                             const float* src = base + (size_t)(2 * c) * slot_elems + (size_t)m0 * kTileCols;
 #pragma unroll
                             for (int q = 0; q < kStep; ++q) acc[q] += __ldcg(src + (size_t)q * kTileCols);
