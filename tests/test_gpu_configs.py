@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2601_16536_b200 import binding as B
 from paper_2601_16536_b200 import workloads as wl
-from gpu_util import assert_close, c_f64, ensure_ws, pack_problem, to_dev
+from gpu_util import assert_close, c_bits, c_f64, ensure_ws, pack_problem, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -57,4 +57,30 @@ def test_results_do_not_depend_on_the_path():
         C = B.w4a16_gemm(A, pw, path=path)
         torch.cuda.synchronize()
         assert_close(c_f64(C), ref, "path %d" % path)
+    del ws
+
+
+@pytest.mark.parametrize("M,path", [(1, B.PATH_TILE), (16, B.PATH_TILE), (32, B.PATH_TILE), (64, B.PATH_TILE),
+                                    (1, B.PATH_DECODE), (8, B.PATH_DECODE)])
+def test_long_k_back_to_back_calls_repeat_bit_for_bit(M, path):
+    # Config 3's shape gives every CTA about a hundred pipeline stages, several segments and
+    # Split-K partial tiles.  Thirty calls queued back to back (each starts while the one before
+    # it drains) must all finish cleanly and produce the very same bits: the order of every sum is
+    # fixed, so any difference means a pipeline hand-off went wrong.  Sampled columns are checked
+    # against the oracle as well.
+    K, N = 28672, 8192
+    d, pw = _packed(next(c for c in _CASES if c.K == K and c.N == N))
+    A_bits = wl.draw_activations(M, K, 99 + M, 1.0, 0)
+    A = to_dev(A_bits)
+    ws = ensure_ws(M, N, K, 0)
+    outs = [B.w4a16_gemm(A, pw, path=path) for _ in range(30)]
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    first = c_bits(outs[0])
+    for i, C in enumerate(outs[1:], 1):
+        assert np.array_equal(c_bits(C), first), "call %d differs from call 0" % i
+    got = c_f64(outs[0])
+    for n0 in (0, 126, N - 4):
+        ref = oracle.gemm(A_bits, d["Wq"], d["S"], d["Z"], M, N, K, 128, cols=(n0, n0 + 4))
+        assert_close(got[:, n0:n0 + 4], ref[:, n0:n0 + 4], "M%d path %d cols %d" % (M, path, n0))
     del ws
