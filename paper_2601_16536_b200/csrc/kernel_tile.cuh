@@ -29,19 +29,21 @@
 // bit-identical from run to run.
 //
 // One pipeline stage is a whole group (128 k, eight MMAs) for batch tiles of up to 64 rows and half
-// a group (64 k, four MMAs) above: narrow tiles are bound by the per-stage hand-offs and by the
-// issuing lane (about 40 clocks per tcgen05.mma whatever its size), wide ones by the tensor pipe.
+// a group (64 k, four MMAs) above: narrow tiles are bound by per-stage work other than the MMAs
+// (the dequant warps' instruction streams, the control warps' loops), wide ones by the tensor pipe.
 // A ring of R slots holds, per slot, the stage's activation boxes in shared memory and its
 // dequantized weights in tensor memory (32 or 64 columns; six or eight slots fit beside the
 // accumulators); the MMAs of a stage release both with one commit.  Four sets of four dequant
 // warps take stages round-robin; inside a set warp w owns TMEM lanes 32 (w % 4) .. + 31.  Each
 // thread keeps the packed words of its next two or three stages in registers (loads issued that
-// far ahead, pointers stepped, no register copies).  With MT <= 128 two accumulators alternate
-// between segments, so one drains while the next fills.  The packed weights do not depend on the
+// far ahead, pointers stepped, no register copies).  Tiles of up to 32 rows have three MMA-issuing
+// warps that take the stages round-robin, each summing into an accumulator of its own (the epilogue
+// adds them in stage order); the others have one issuer, and two accumulators that alternate
+// between segments (MT = 16, 64, 128), so one drains while the next fills.  The packed weights do not depend on the
 // previous kernel in the stream: under programmatic dependent launch the dequant warps load and
 // convert weights until the TMEM ring is full before anything waits for that kernel; only
 // activations, C and the workspace are touched after griddepcontrol.wait.
-// The producer and MMA warps run warp-uniform loops and elect one lane per instruction, which
+// The producer and issuer warps run warp-uniform loops and elect one lane per instruction, which
 // keeps descriptors in uniform registers.  All waits are bounded mbarrier waits; a wait that runs
 // out records a status code and the CTA drains and exits (TMEM is always released).
 //
@@ -560,8 +562,11 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                 n_prev = n;
                 // convert ring slot pi, then refill it with the stage kPF ahead
                 if (pi == 0) { ok = convert(pf0, n); fetch(pf0); pi = 1; }
-                else if (pi == 1) { ok = convert(pf1, n); fetch(pf1); pi = (kPF == 3) ? 2 : 0; }
-                else { ok = convert(pf2, n); fetch(pf2); pi = 0; }
+                else if (kPF == 2 || pi == 1) { ok = convert(pf1, n); fetch(pf1); pi = (kPF == 3) ? 2 : 0; }
+                else {
+                    if constexpr (kPF == 3) { ok = convert(pf2, n); fetch(pf2); }
+                    pi = 0;
+                }
                 if (!ok) break;
                 tc_wait_st();
                 tc_fence_before();
