@@ -25,7 +25,7 @@ struct DeviceState {
     int max_smem_optin = 0;
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    bool decode_attr_set[3] = {false, false, false};
+    bool decode_attr_set[3][4] = {};   // [mb][CTAs per SM]
     bool tile_attr_set[5] = {false, false, false, false, false};
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
     // kernel in its stream has finished.  After w4a16_pack was enqueued the next GEMM launch is
@@ -78,10 +78,12 @@ int sm_count_or_default() {
 // ---- decode-path launch geometry ------------------------------------------------
 int decode_mb(int M) { return M <= 8 ? 1 : 2; }
 
-// The decode kernel is persistent: `ctas` CTAs per batch chunk (two per SM: 9 warps and about
-// 100 KiB of shared memory each), `nchunks` chunks of work units dealt to them.
+// The decode kernel is persistent: `ctas` CTAs per batch chunk (two per SM with about 100 KiB of
+// shared memory each, or three with about 60 KiB; 9 warps), `nchunks` chunks of work units dealt to
+// them.
 struct DecodeGeom {
     int mb, mchunks, stages, smem_bytes, ctas, nchunks;
+    int cps;       // CTAs per SM the launch is sized for (2 or 3)
     int split_k;   // what the kernel runs: 0 = balanced chunks, S >= 1 = S slices per tile
 };
 
@@ -91,13 +93,18 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms) {
     g.mchunks = (M + 8 * g.mb - 1) / (8 * g.mb);
     const int T = N / kTileN;
     const long units = (long)T * G;
-    const int budget = (227 * 1024) / 2 - 1024;   // per CTA, two CTAs per SM
+    // Three CTAs per SM (a two-stage ring each) when every CTA has a long stream: measured with one
+    // batch block, 34.3 against 36.7 us at K = 28672 / N = 8192, 18.1 against 18.9 at K = 4096 /
+    // N = 22016, 12.6 against 13.5 at N = 12288, but 12.3 against 11.9 at K = 11008 / N = 4096 and
+    // 8.0 against 7.1 at K = N = 4096.  Two batch blocks leave room for one stage only: two CTAs.
+    g.cps = (g.mb == 1 && units >= 20L * 2 * sms) ? 3 : 2;
+    const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
     int st = (budget - 128 - decode_red_bytes(g.mb)) / decode_stage_bytes(g.mb);
     if (st > kDecMaxStages) st = kDecMaxStages;
     if (st < 2) st = 2;
     g.stages = st;
     g.smem_bytes = decode_smem_bytes(g.mb, st);
-    long slots = 2L * sms;
+    long slots = (long)g.cps * sms;
     if (split_k == 0 && T <= slots) {
         // Balanced chunks use every CTA slot, but a chunk that crosses a tile boundary goes through the
         // partial-tile exchange in mid-stream (about six units' worth of time).  S slices per tile keep
@@ -525,14 +532,14 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    auto kern = (g.mb == 1) ? gemm_decode_kernel<1> : gemm_decode_kernel<2>;
-    if (!d->decode_attr_set[g.mb]) {
+    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2> : (g.cps == 3) ? gemm_decode_kernel<1, 3> : gemm_decode_kernel<1, 2>;
+    if (!d->decode_attr_set[g.mb][g.cps]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
         }
-        d->decode_attr_set[g.mb] = true;
+        d->decode_attr_set[g.mb][g.cps] = true;
     }
     // programmatic dependent launch (see the tile path above): prologue and weight prefetch may overlap
     // the tail of the previous kernel in the stream
@@ -627,14 +634,14 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    auto kern = (g.mb == 1) ? gemm_decode_kernel<1> : gemm_decode_kernel<2>;
-    if (!d->decode_attr_set[g.mb]) {
+    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2> : (g.cps == 3) ? gemm_decode_kernel<1, 3> : gemm_decode_kernel<1, 2>;
+    if (!d->decode_attr_set[g.mb][g.cps]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
         }
-        d->decode_attr_set[g.mb] = true;
+        d->decode_attr_set[g.mb][g.cps] = true;
     }
     kern<<<dim3(g.ctas, g.mchunks, 1), kDecThreads, g.smem_bytes, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;

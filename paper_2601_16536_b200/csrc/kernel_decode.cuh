@@ -123,9 +123,12 @@ struct DecStageIter {
     }
 };
 
-// MB = number of 8-row batch blocks one CTA handles (rows m0 .. m0 + 8 MB - 1).
-template <int MB>
-__global__ void __launch_bounds__(kDecThreads) gemm_decode_kernel(const DecodeParams p) {
+// MB = number of 8-row batch blocks one CTA handles (rows m0 .. m0 + 8 MB - 1).  CPS = CTAs the
+// launch wants resident per SM (2, or 3 with a two-stage ring and at most 72 registers: more warps
+// per scheduler pay on long launches, the shallower ring and the extra Split-K slices cost on short
+// ones; the host picks, see decode_geom).
+template <int MB, int CPS>
+__global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kRows = 8 * MB;
     const int mz = blockIdx.y;
