@@ -25,7 +25,7 @@ struct DeviceState {
     int max_smem_optin = 0;
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    bool decode_attr_set[3][4] = {};   // [mb][CTAs per SM]
+    bool decode_attr_set[3][4][2] = {};   // [mb][CTAs per SM][cluster exchange]
     bool tile_attr_set[5] = {false, false, false, false, false};
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
     // kernel in its stream has finished.  After w4a16_pack was enqueued the next GEMM launch is
@@ -84,10 +84,11 @@ int decode_mb(int M) { return M <= 8 ? 1 : 2; }
 struct DecodeGeom {
     int mb, mchunks, stages, smem_bytes, ctas, nchunks;
     int cps;       // CTAs per SM the launch is sized for (2 or 3)
+    bool cluster;  // one thread-block cluster of split_k CTAs per tile: partial tiles meet in shared memory
     int split_k;   // what the kernel runs: 0 = balanced chunks, S >= 1 = S slices per tile
 };
 
-DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms) {
+DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_cluster = true) {
     DecodeGeom g;
     g.mb = decode_mb(M);
     g.mchunks = (M + 8 * g.mb - 1) / (8 * g.mb);
@@ -98,12 +99,6 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms) {
     // N = 22016, 12.6 against 13.5 at N = 12288, but 12.3 against 11.9 at K = 11008 / N = 4096 and
     // 8.0 against 7.1 at K = N = 4096.  Two batch blocks leave room for one stage only: two CTAs.
     g.cps = (g.mb == 1 && units >= 20L * 2 * sms) ? 3 : 2;
-    const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
-    int st = (budget - 128 - decode_red_bytes(g.mb)) / decode_stage_bytes(g.mb);
-    if (st > kDecMaxStages) st = kDecMaxStages;
-    if (st < 2) st = 2;
-    g.stages = st;
-    g.smem_bytes = decode_smem_bytes(g.mb, st);
     long slots = (long)g.cps * sms;
     if (split_k == 0 && T <= slots) {
         // Balanced chunks use every CTA slot, but a chunk that crosses a tile boundary goes through the
@@ -128,6 +123,15 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms) {
         g.nchunks = T * split_k;
         g.ctas = (int)((long)g.nchunks < slots ? (long)g.nchunks : slots);
     }
+    // S slices per tile, every slice on a CTA of its own, one batch chunk: the S CTAs of a tile form a
+    // cluster and exchange their partial tiles through distributed shared memory
+    g.cluster = allow_cluster && split_k >= 2 && split_k <= kDecMaxCluster && g.nchunks == g.ctas && g.mchunks == 1;
+    const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
+    int st = (budget - 128 - decode_red_bytes(g.mb) - decode_xch_bytes(g.mb, g.cluster)) / decode_stage_bytes(g.mb);
+    if (st > kDecMaxStages) st = kDecMaxStages;
+    if (st < 2) st = 2;
+    g.stages = st;
+    g.smem_bytes = decode_smem_bytes(g.mb, st, g.cluster);
     return g;
 }
 
@@ -519,6 +523,7 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count);
     if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
     if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
+    // (the cluster exchange does not touch the workspace, but the contract stays the same for every schedule)
     if (g.split_k != 1 && ws_body_bytes < decode_partial_bytes(g)) return W4A16_ERR_WORKSPACE;
     DecodeParams p;
     p.A = Ah;
@@ -532,14 +537,18 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2> : (g.cps == 3) ? gemm_decode_kernel<1, 3> : gemm_decode_kernel<1, 2>;
-    if (!d->decode_attr_set[g.mb][g.cps]) {
+    void (*kern)(const DecodeParams) =
+        g.cluster ? ((g.mb == 2) ? gemm_decode_kernel<2, 2, true>
+                                 : (g.cps == 3) ? gemm_decode_kernel<1, 3, true> : gemm_decode_kernel<1, 2, true>)
+                  : ((g.mb == 2) ? gemm_decode_kernel<2, 2, false>
+                                 : (g.cps == 3) ? gemm_decode_kernel<1, 3, false> : gemm_decode_kernel<1, 2, false>);
+    if (!d->decode_attr_set[g.mb][g.cps][g.cluster ? 1 : 0]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
         }
-        d->decode_attr_set[g.mb][g.cps] = true;
+        d->decode_attr_set[g.mb][g.cps][g.cluster ? 1 : 0] = true;
     }
     // programmatic dependent launch (see the tile path above): prologue and weight prefetch may overlap
     // the tail of the previous kernel in the stream
@@ -548,11 +557,22 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     cfg.blockDim = dim3(kDecThreads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (g.cluster) {   // the split_k CTAs of a column tile are one cluster (consecutive blockIdx.x)
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = (unsigned)g.split_k;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    if (d->pdl_ok) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = d->pdl_ok ? 1 : 0;
+    cfg.numAttrs = n_attr;
     d->pdl_ok = true;
     if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) {
         cudaGetLastError();
@@ -600,7 +620,7 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return W4A16_ERR_CUDA;
 
-    const DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count);
+    const DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, false);   // no clusters here: this entry point keeps the path it was built with
     if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
     if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
     // the whole scratch need of this shape must fit the built-in array, or nothing is launched
@@ -634,14 +654,15 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2> : (g.cps == 3) ? gemm_decode_kernel<1, 3> : gemm_decode_kernel<1, 2>;
-    if (!d->decode_attr_set[g.mb][g.cps]) {
+    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2, false>
+                            : (g.cps == 3) ? gemm_decode_kernel<1, 3, false> : gemm_decode_kernel<1, 2, false>;
+    if (!d->decode_attr_set[g.mb][g.cps][0]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
         }
-        d->decode_attr_set[g.mb][g.cps] = true;
+        d->decode_attr_set[g.mb][g.cps][0] = true;
     }
     kern<<<dim3(g.ctas, g.mchunks, 1), kDecThreads, g.smem_bytes, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;

@@ -111,6 +111,31 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return false;
 }
 
+// The same bounded wait with cluster-scope acquire: for a barrier that CTAs of the cluster arrive on
+// after writing this CTA's shared memory.
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    unsigned long long t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (;;) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
+            : "memory");
+        if (ok) return true;
+        unsigned long long t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        if (t1 - t0 > 2000000000ull) break;
+    }
+    report_status(kStatusMbarTimeout);
+    return false;
+}
+
 // One lane of a converged warp (warp-uniform control flow keeps addresses and descriptors in
 // uniform registers; only the issuing instruction itself is predicated on the elected lane).
 __device__ __forceinline__ bool elect_one() {

@@ -61,8 +61,11 @@ __host__ __device__ inline int decode_stage_bytes(int mb) { return kDecStageA + 
 __host__ __device__ inline int decode_red_bytes(int mb) {
     return kDecUnitsPerStage * 8 * mb * kDecRedStride * 4;
 }
-__host__ __device__ inline int decode_smem_bytes(int mb, int stages) {
-    return 128 + decode_red_bytes(mb) + stages * decode_stage_bytes(mb);
+// cluster exchange buffer (CL kernels): up to kDecMaxCluster partial tiles of 8 mb rows x 64 columns
+constexpr int kDecMaxCluster = 4;
+__host__ __device__ inline int decode_xch_bytes(int mb, bool cl) { return cl ? kDecMaxCluster * 8 * mb * kTileN * 4 : 0; }
+__host__ __device__ inline int decode_smem_bytes(int mb, int stages, bool cl) {
+    return 128 + decode_red_bytes(mb) + decode_xch_bytes(mb, cl) + stages * decode_stage_bytes(mb);
 }
 
 // D += A . B with A = (a0: row gq, a1: row gq + 8, a2 / a3: the same rows, second k pair).
@@ -127,7 +130,12 @@ struct DecStageIter {
 // launch wants resident per SM (2, or 3 with a two-stage ring and at most 72 registers: more warps
 // per scheduler pay on long launches, the shallower ring and the extra Split-K slices cost on short
 // ones; the host picks, see decode_geom).
-template <int MB, int CPS>
+// CL: the launch is made of thread-block clusters of split_k CTAs, one cluster per column tile and
+// one K slice per CTA (classic Split-K, every chunk on a CTA of its own).  The slices' partial tiles
+// then meet in the shared memory of the cluster's first CTA (distributed shared memory + one
+// hardware cluster barrier) instead of going through the workspace, a fence, a ticket and a reload:
+// Phase 3 of Algorithm 1 in about a tenth of the time, still summed in ascending K order.
+template <int MB, int CPS, bool CL>
 __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kRows = 8 * MB;
@@ -141,20 +149,31 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
     // shared layout: [barriers + flag, 128 B][reduce buffer][stage 0][stage 1]...
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);
     uint64_t* empty = full + kDecMaxStages;
+    uint64_t* xbar = full + 2 * kDecMaxStages;   // CL only: the slices' partial tiles have landed (CTA 0's is used)
     int* last_flag = reinterpret_cast<int*>(smem + 120);
     float* red = reinterpret_cast<float*>(smem + 128);
-    unsigned char* stage0 = smem + 128 + decode_red_bytes(MB);
+    float* xch = reinterpret_cast<float*>(smem + 128 + decode_red_bytes(MB));   // CL only: [slice][8 MB rows][64]
+    unsigned char* stage0 = smem + 128 + decode_red_bytes(MB) + decode_xch_bytes(MB, CL);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
             mbar_init(&full[i], 1);
             mbar_init(&empty[i], kDecWarps);
         }
+        if (CL) mbar_init(xbar, (uint32_t)(p.split_k * kDecWarps));   // one arrival per consumer warp of the cluster
         fence_mbar_init();
     }
     // (Batch rows this CTA does not have are never loaded: an MMA column only feeds its own output
     // column, and those columns are not stored.)
     __syncthreads();
+    // CL: every CTA of the cluster is running and has initialised its barriers before anyone writes to
+    // another CTA's shared memory.  All threads of all CTAs of the cluster pass here unconditionally
+    // (the hardware launches a cluster's CTAs together); every later wait in this kernel is a bounded
+    // mbarrier wait.
+    if (CL) {
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
     // Let the next kernel in the stream start its own prologue and weight prefetch; everything below
     // that reads or writes memory another kernel may have written comes after griddepcontrol.wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -325,6 +344,35 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
             const bool whole = (seg_start == tile_u0) && (u == tile_end);
             // first segment of a chunk -> slot 2 ci, a chunk's continuation into a later tile -> 2 ci + 1
             float* my_slot = ws_mz + (size_t)(2 * ci + (seg_start == u0 ? 0 : 1)) * (kRows * kTileN);
+            if (CL && !whole) {
+                // this CTA's slice -> slot `rank` of the exchange buffer of the cluster's CTA 0
+                uint32_t rank, xch0, xbar0;
+                asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xch0) : "r"(smem_u32(xch)), "r"(0u));
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xbar0) : "r"(smem_u32(xbar)), "r"(0u));
+                for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
+                    const int n = idx & (kTileN - 1), m = idx >> 6;
+                    float v = red[m * kDecRedStride + n];
+#pragma unroll
+                    for (int w = 1; w < kDecUnitsPerStage; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
+                    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(xch0 + (rank * (kRows * kTileN) + idx) * 4u), "f"(v)
+                                 : "memory");
+                }
+                // the warp's stores, then one release-arrival per warp on CTA 0's barrier
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(xbar0) : "memory");
+                if (rank == 0) {
+                    if (!mbar_wait_cluster(xbar, 0u)) return;   // status recorded
+                    for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
+                        const int n = idx & (kTileN - 1), m = idx >> 6;
+                        float v = xch[idx];
+                        for (int sl = 1; sl < p.split_k; ++sl) v += xch[sl * (kRows * kTileN) + idx];
+                        p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
+                    }
+                }
+                return;   // one slice per CTA: nothing follows
+            }
             for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
                 const int n = idx & (kTileN - 1), m = idx >> 6;
                 float v = red[m * kDecRedStride + n];
