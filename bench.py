@@ -37,7 +37,10 @@ PATH_NAMES = {1: "gemm_simple_kernel", 2: "gemm_decode_kernel", 3: "gemm_tile_ke
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until captured)
-NCU_TRAFFIC_BYTES = 24134016           # gemm_tile_kernel<16>, M=16 K=11008 N=4096 (read 24.13 MB, write 0)
+# DRAM read + write of one M=16 K=11008 N=4096 launch, by the kernel the library picks for it (ncu; None = not
+# captured since that kernel last changed)
+NCU_TRAFFIC_BYTES = {"gemm_tile_kernel": 24134016,      # read 24.13 MB, write 0
+                     "gemm_decode_kernel": 23817984}    # read 23.82 MB, write 0 (<2, 2, cluster>)
 NCU_TRAFFIC_BYTES_TILE = 194827776    # gemm_tile_kernel<256>, M=4096 K=N=8192 (read 135.8 MB + write 59.1 MB)
 
 
@@ -400,9 +403,10 @@ def run_ours(args):
     dom_M = SWEEP_M[-1]
     dom_bytes = wl.algorithmic_bytes(dom_M, K, N)
     achieved = dom_bytes / per_call[dom_M] / 1e9
-    roofline = {"bound": "hbm", "kernel": PATH_NAMES.get(B.w4a16_choose_path(dom_M, N, K), "?"), "case": "M=%d K=%d N=%d" % (dom_M, K, N),
+    dom_kernel = PATH_NAMES.get(B.w4a16_choose_path(dom_M, N, K), "?")
+    roofline = {"bound": "hbm", "kernel": dom_kernel, "case": "M=%d K=%d N=%d" % (dom_M, K, N),
                 "achieved": achieved, "peak": hbm_peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES,
+                "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES.get(dom_kernel),
                 "algorithmic_bytes_per_launch": dom_bytes,
                 "launch_us": per_call[dom_M] * 1e6,
                 "sweep_frac": value / world / hbm_peak}

@@ -275,12 +275,17 @@ bool make_act_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mt) 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Path taken when the caller does not force one.  Measured on B200 (K = 11008, N = 4096 and K = 28672,
-// N = 8192): up to 8 batch rows the warp-MMA kernel is ahead (13.7 us against 14.6 us), from 9 rows on
-// it needs a second batch block per weight and the tcgen05 kernel wins (14.8 us against 17.8 us at 16).
-int resolve_path(int M, int path) {
-    if (path == W4A16_PATH_AUTO) return M > 8 ? W4A16_PATH_TILE : W4A16_PATH_DECODE;
-    return path;
+// Path taken when the caller does not force one.  Measured on B200: up to 8 batch rows the warp-MMA
+// kernel is ahead everywhere (K = 11008 / N = 4096: 9.8 us against 12.9; K = 28672 / N = 8192: 34 against
+// 44).  From 9 to 16 rows it needs a second batch block per weight; it still wins where its K slices
+// exchange through a cluster (M = 16: 12.5 against 12.9 us at K = 11008 / N = 4096, 6.9 against 8.6 at
+// K = N = 4096) and loses where they cannot (16.9 against 16.5 at N = 12288, 46.3 against 44.7 at
+// K = 28672 / N = 8192).  Above 16 rows the tcgen05 kernel.
+int resolve_path(int M, int N, int G, int split_k, int sms, int path) {
+    if (path != W4A16_PATH_AUTO) return path;
+    if (M <= 8) return W4A16_PATH_DECODE;
+    if (M <= 16 && decode_geom(M, N, G, split_k, sms).cluster) return W4A16_PATH_DECODE;
+    return W4A16_PATH_TILE;
 }
 
 // FP32 partials of the two-kernel reduce used by the plain path: [split_k][M][N].
@@ -336,7 +341,7 @@ size_t w4a16_packed_z_bytes(int N, int K, int group) {
 int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return 1;
     int G = K / group;
-    switch (resolve_path(M, path)) {
+    switch (resolve_path(M, N, G, 0, sm_count_or_default(), path)) {
         case W4A16_PATH_DECODE: return choose_split_decode(M, N, G, sm_count_or_default());
         case W4A16_PATH_TILE: return choose_split_tile(M, N, G, sm_count_or_default());
         default: return 1;
@@ -344,7 +349,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
 }
 int w4a16_choose_path(int M, int N, int K, int group) {
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return W4A16_ERR_SHAPE;
-    return resolve_path(M, W4A16_PATH_AUTO);
+    return resolve_path(M, N, K / group, 0, sm_count_or_default(), W4A16_PATH_AUTO);
 }
 int w4a16_choose_split_k(int M, int N, int K, int group) {
     return w4a16_choose_split_k_ex(M, N, K, group, W4A16_PATH_AUTO);
@@ -438,7 +443,7 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     if ((rc = current_device(&d)) != W4A16_OK) return rc;
     if (!d->is_sm100) return W4A16_ERR_ARCH;
 
-    path = resolve_path(M, path);
+    path = resolve_path(M, N, G, split_k, d->sm_count, path);
     if (split_k > 65535) return W4A16_ERR_SPLITK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __half* Ah = reinterpret_cast<const __half*>(A);
