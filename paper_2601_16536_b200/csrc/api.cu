@@ -32,6 +32,7 @@ struct DeviceState {
     // therefore a plain, fully ordered one (it runs after the pack kernels), and only the launches
     // after it overlap their predecessor again.
     bool pdl_ok = false;
+    bool cluster_ok = true;   // cleared when a cluster launch is refused (fewer SMs than usual, MPS limits ...)
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -73,6 +74,12 @@ int sm_count_or_default() {
     DeviceState* d = nullptr;
     if (current_device(&d) == W4A16_OK) return d->sm_count;
     return 148;
+}
+
+bool cluster_ok_or_default() {
+    DeviceState* d = nullptr;
+    if (current_device(&d) == W4A16_OK) return d->cluster_ok;
+    return true;
 }
 
 // ---- decode-path launch geometry ------------------------------------------------
@@ -281,10 +288,10 @@ bool make_act_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mt) 
 // exchange through a cluster (M = 16: 12.5 against 12.9 us at K = 11008 / N = 4096, 6.9 against 8.6 at
 // K = N = 4096) and loses where they cannot (16.9 against 16.5 at N = 12288, 46.3 against 44.7 at
 // K = 28672 / N = 8192).  Above 16 rows the tcgen05 kernel.
-int resolve_path(int M, int N, int G, int split_k, int sms, int path) {
+int resolve_path(int M, int N, int G, int split_k, int sms, int path, bool allow_cluster = true) {
     if (path != W4A16_PATH_AUTO) return path;
     if (M <= 8) return W4A16_PATH_DECODE;
-    if (M <= 16 && decode_geom(M, N, G, split_k, sms).cluster) return W4A16_PATH_DECODE;
+    if (M <= 16 && decode_geom(M, N, G, split_k, sms, allow_cluster).cluster) return W4A16_PATH_DECODE;
     return W4A16_PATH_TILE;
 }
 
@@ -341,7 +348,7 @@ size_t w4a16_packed_z_bytes(int N, int K, int group) {
 int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return 1;
     int G = K / group;
-    switch (resolve_path(M, N, G, 0, sm_count_or_default(), path)) {
+    switch (resolve_path(M, N, G, 0, sm_count_or_default(), path, cluster_ok_or_default())) {
         case W4A16_PATH_DECODE: return choose_split_decode(M, N, G, sm_count_or_default());
         case W4A16_PATH_TILE: return choose_split_tile(M, N, G, sm_count_or_default());
         default: return 1;
@@ -349,7 +356,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
 }
 int w4a16_choose_path(int M, int N, int K, int group) {
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return W4A16_ERR_SHAPE;
-    return resolve_path(M, N, K / group, 0, sm_count_or_default(), W4A16_PATH_AUTO);
+    return resolve_path(M, N, K / group, 0, sm_count_or_default(), W4A16_PATH_AUTO, cluster_ok_or_default());
 }
 int w4a16_choose_split_k(int M, int N, int K, int group) {
     return w4a16_choose_split_k_ex(M, N, K, group, W4A16_PATH_AUTO);
@@ -443,7 +450,8 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     if ((rc = current_device(&d)) != W4A16_OK) return rc;
     if (!d->is_sm100) return W4A16_ERR_ARCH;
 
-    path = resolve_path(M, N, G, split_k, d->sm_count, path);
+    const int path_asked = path;
+    path = resolve_path(M, N, G, split_k, d->sm_count, path, d->cluster_ok);
     if (split_k > 65535) return W4A16_ERR_SPLITK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __half* Ah = reinterpret_cast<const __half*>(A);
@@ -525,7 +533,7 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     }
 
     // W4A16_PATH_DECODE
-    DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count);
+    DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, d->cluster_ok);
     if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
     if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
     // (the cluster exchange does not touch the workspace, but the contract stays the same for every schedule)
@@ -581,6 +589,12 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     d->pdl_ok = true;
     if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) {
         cudaGetLastError();
+        if (g.cluster) {
+            // the device would not place the clusters: from now on the workspace exchange (and the path
+            // rule that goes with it), starting with this call
+            d->cluster_ok = false;
+            return w4a16_gemm_ex(A, Wq, S, Z, C, M, N, K, group, split_k, path_asked, stream);
+        }
         return W4A16_ERR_CUDA;
     }
     return W4A16_OK;
