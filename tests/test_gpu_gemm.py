@@ -139,3 +139,24 @@ def test_host_buffer_entry_point_matches_device_call():
     C = B.w4a16_gemm(to_dev(d["A"]), pw)
     assert np.array_equal(C_host.numpy().view(np.uint16), c_bits(C))
     del ws
+
+
+@pytest.mark.parametrize("M,split_k", [(1, 2), (5, 4), (8, 3), (16, 4), (12, 0)])
+def test_cluster_exchange_and_workspace_exchange_give_the_same_bits(M, split_k):
+    # Algorithm 1, Phase 3 in its two forms: w4a16_gemm on the warp-MMA path adds the slices of a tile
+    # inside a thread-block cluster when each slice has a CTA of its own; w4a16_gemm_static_ws keeps
+    # the workspace form (partial tiles, tickets, last arriver).  Both add in ascending K order, so
+    # the outputs must agree bit for bit, and with the oracle within tolerance.
+    K, N = 4096, 1024
+    d = wl.make_problem(M, K, N, seed=600 + M)
+    pw = pack_problem(d, N, K)
+    A = to_dev(d["A"])
+    ws = ensure_ws(M, N, K, split_k)
+    got = B.w4a16_gemm(A, pw, split_k=split_k, path=B.PATH_DECODE)
+    other = B.w4a16_gemm_static_ws(A, pw, split_k=split_k)
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    assert np.array_equal(c_bits(got), c_bits(other))
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+    assert_close(c_f64(got), ref, "M%d split %d" % (M, split_k))
+    del ws
