@@ -109,14 +109,17 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     long slots = (long)g.cps * sms;
     if (split_k == 0 && T <= slots) {
         // Balanced chunks use every CTA slot, but a chunk that crosses a tile boundary goes through the
-        // partial-tile exchange in mid-stream (about six units' worth of time).  S slices per tile keep
-        // every chunk inside one tile at the price of idle slots.  Take the cheaper (units per CTA;
-        // measured: K = 11008 / N = 4096 and K = N = 4096 gain 8-23 % from slices, K = 28672 / N = 8192
-        // loses 5 %).
+        // workspace exchange in mid-stream.  S slices per tile keep every chunk inside one tile at the
+        // price of idle slots, and their exchange is cheaper: none at S = 1, through the cluster for
+        // S <= 4, at the end of the stream otherwise.  Costs in units per CTA, the exchanges priced from
+        // measurements (K = 4096 / N = 22016, M = 1: whole tiles 16.0 us against 18.4 balanced;
+        // K = 28672 / N = 8192: three slices 35.1 against 35.0; K = 11008 / N = 4096: four slices 9.8
+        // against 11.9 before there were clusters).
         int s0 = (int)(slots / T);
         if (s0 > G) s0 = G;
-        const long classic_cost = (G + s0 - 1) / s0;
-        const long balanced_cost = (units + slots - 1) / slots + 6;
+        const bool clusterable = allow_cluster && s0 >= 2 && s0 <= kDecMaxCluster && g.mchunks == 1;
+        const long classic_cost = (G + s0 - 1) / s0 + (s0 == 1 ? 0 : clusterable ? 4 : 6);
+        const long balanced_cost = (units + slots - 1) / slots + 12;
         if (classic_cost <= balanced_cost) split_k = s0;
     }
     g.split_k = split_k;
