@@ -364,6 +364,12 @@ def run_ours(args):
                "us": sec * 1e6, "eff_GBps": byts / sec / 1e9, "tflops": fl / sec / 1e12,
                "bound": "tensor" if fl / (tc_peak * 1e12) > byts / (hbm_peak * 1e9) else "hbm",
                "roofline_frac": max(byts / (hbm_peak * 1e9), fl / (tc_peak * 1e12)) / sec}
+        if c.config == 6:
+            # the paper's Figure 2 comparison: one slice ("data parallel") beside the chosen schedule
+            sec1 = _time_calls(lambda: B.w4a16_gemm(A, cur.take(), C, split_k=1), 5,
+                               max(20, args.case_calls // 8), torch)
+            rec["us_split_k_1"] = sec1 * 1e6
+            rec["splitk_speedup"] = sec1 / sec
         if not args.no_cublas:
             if cur_w16 is None:
                 ncopy = max(2, min(6, (MIN_ROTATION_BYTES // 2) // (c.K * c.N * 2) + 1))
@@ -527,7 +533,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--split-k", type=int, default=0, help="force one split factor (0 = automatic)")
-    ap.add_argument("--configs", type=lambda s: [int(x) for x in s.split(",")], default=[1, 3, 4, 5],
+    ap.add_argument("--configs", type=lambda s: [int(x) for x in s.split(",")], default=[1, 3, 4, 5, 6],
                     help="besides the timed config-2 step, report every case of these configs (2 = none)")
     ap.add_argument("--case-calls", type=int, default=400)
     ap.add_argument("--no-cublas", action="store_true")

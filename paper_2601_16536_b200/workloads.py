@@ -24,9 +24,13 @@ import numpy as np
 GROUP = 128
 
 
+# (N, K) of the layers the paper measures (Figure 2 a-f; its "K = 16348" is read as 16384)
+PAPER_SHAPES = ((1536, 6144), (2048, 8192), (2048, 10240), (4096, 16384), (4608, 10240), (7168, 18432))
+
+
 @dataclass(frozen=True)
 class Case:
-    config: int       # 1..5, the benchmark configuration the case belongs to
+    config: int       # 1..5, the benchmark configuration the case belongs to; 6 = the paper's own shapes
     name: str
     M: int
     K: int
@@ -51,6 +55,12 @@ def _cases() -> List[Case]:
             i += 1
     for i, M in enumerate((256, 1024, 4096)):
         out.append(Case(5, "prefill_8192", M, 8192, 8192, 5000 + i))
+    # the paper's own shape set (Section 4.1, Figure 2: six (N, K) pairs, batch sizes up to 256)
+    i = 0
+    for N, K in PAPER_SHAPES:
+        for M in (1, 8, 64, 256):
+            out.append(Case(6, "paper_N%d_K%d" % (N, K), M, K, N, 6000 + i))
+            i += 1
     return out
 
 

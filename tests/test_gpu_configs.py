@@ -1,5 +1,6 @@
-"""GPU parity at the benchmark's full sizes (configs 1-4), in the launch configuration bench.py
-times: automatic path, automatic split.  The oracle (Eq. 2 in FP64) computes whole columns of C,
+"""GPU parity at the benchmark's full sizes (configs 1-4, and the paper's own shape set of
+Section 4.1 / Figure 2 as config 6), in the launch configuration bench.py times: automatic path,
+automatic split.  The oracle (Eq. 2 in FP64) computes whole columns of C,
 sampled at tile edges, a tile interior and the last columns; all rows of the batch are checked."""
 import numpy as np
 import pytest
@@ -12,7 +13,7 @@ from gpu_util import assert_close, c_bits, c_f64, ensure_ws, pack_problem, to_de
 
 pytestmark = pytest.mark.gpu
 
-_CASES = [c for c in wl.CASES if c.config in (1, 2, 3, 4)]
+_CASES = [c for c in wl.CASES if c.config in (1, 2, 3, 4, 6)]
 _weights = {}
 
 
