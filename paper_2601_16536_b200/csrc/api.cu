@@ -170,11 +170,29 @@ constexpr size_t kTileTicketBytes = 131072;   // 16 counters per tile, after the
 constexpr size_t kWsFullHeaderBytes = kWsHeaderBytes + kTileTicketBytes;
 constexpr long kTileMaxTicketTiles = kTileTicketBytes / (sizeof(int) * kTileDequantWarps);
 
-int tile_mt_index(int M) { return M <= 16 ? 0 : M <= 32 ? 1 : M <= 64 ? 2 : M <= 128 ? 3 : 4; }
+// Batch rows per CTA tile: the smallest of 16 .. 256 that covers M -- except that a narrow weight
+// matrix gives such tiles too few of them for 148 SMs (N = 1536 and M = 256: twelve), and the
+// twelve-way Split-K that follows costs more than converting the weights once per narrower batch tile.
+// With 24 tiles or fewer, take the widest narrower tile that gives at least 24 (never 128 rows, which
+// measured slower than 64 everywhere it was tried).  Measured: M = 256, K = 6144 / N = 1536: 42.5 us
+// with 256-row tiles, 14.8 with 64 (torch FP16 matmul 16.7); M = 256, K = 8192 / N = 2048: 38.3 against
+// 19.9; M = 64, N = 1536: 14.5 against 10.1 with 32 rows; M = 32: 10.7 against 9.0 with 16.  From N = 4096
+// on (32 column tiles) the covering tile wins (M = 256, K = 16384: 41.8 against 52.4 us).
+int tile_mt_index(int M, int N) {
+    const int idx = M <= 16 ? 0 : M <= 32 ? 1 : M <= 64 ? 2 : M <= 128 ? 3 : 4;
+    const long n_tiles = (N + kTileCols - 1) / kTileCols;
+    auto tiles = [&](int i) { return (long)((M + (16 << i) - 1) / (16 << i)) * n_tiles; };
+    if (tiles(idx) > 24) return idx;
+    for (int i = idx - 1; i >= 0; --i) {
+        if (i == 3) continue;
+        if (tiles(i) >= 24) return i;
+    }
+    return 0;   // even 16-row tiles are few: take the most there are
+}
 
 TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
     TileGeom g;
-    g.mt_index = tile_mt_index(M);
+    g.mt_index = tile_mt_index(M, N);
     g.mt = 16 << g.mt_index;
     g.m_tiles = (M + g.mt - 1) / g.mt;
     g.n_tiles = (N + kTileCols - 1) / kTileCols;
