@@ -111,16 +111,25 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
         // Balanced chunks use every CTA slot, but a chunk that crosses a tile boundary goes through the
         // workspace exchange in mid-stream.  S slices per tile keep every chunk inside one tile at the
         // price of idle slots, and their exchange is cheaper: none at S = 1, through the cluster for
-        // S <= 4, at the end of the stream otherwise.  Costs in units per CTA, the exchanges priced from
+        // S <= 6, at the end of the stream otherwise.  Costs in units per CTA, the exchanges priced from
         // measurements (K = 4096 / N = 22016, M = 1: whole tiles 16.0 us against 18.4 balanced;
         // K = 28672 / N = 8192: three slices 35.1 against 35.0; K = 11008 / N = 4096: four slices 9.8
-        // against 11.9 before there were clusters).
+        // against 11.9 before there were clusters; K = 6144 / N = 1536: six slices in a cluster 4.8
+        // against 6.5 for twelve through the workspace).
         int s0 = (int)(slots / T);
         if (s0 > G) s0 = G;
-        const bool clusterable = allow_cluster && s0 >= 2 && s0 <= kDecMaxCluster && g.mchunks == 1;
-        const long classic_cost = (G + s0 - 1) / s0 + (s0 == 1 ? 0 : clusterable ? 4 : 6);
-        const long balanced_cost = (units + slots - 1) / slots + 12;
-        if (classic_cost <= balanced_cost) split_k = s0;
+        // exchange prices in units: none 0, cluster 4, workspace at the end of a slice 9, workspace in
+        // mid-stream (balanced chunks) 13 -- 1.3 / 2.8 / about 4 us at 0.3 us per unit
+        long best = (units + slots - 1) / slots + 13;
+        int best_s = 0;
+        const long ws_cost = (G + s0 - 1) / s0 + (s0 == 1 ? 0 : 9);
+        if (ws_cost <= best) { best = ws_cost; best_s = s0; }
+        if (allow_cluster && g.mchunks == 1 && s0 >= 2) {
+            const int sc = s0 < kDecMaxCluster ? s0 : kDecMaxCluster;   // fewer, longer slices that fit a cluster
+            const long cl_cost = (G + sc - 1) / sc + 4;
+            if (cl_cost <= best) { best = cl_cost; best_s = sc; }
+        }
+        split_k = best_s;
     }
     g.split_k = split_k;
     if (split_k == 0) {
@@ -137,11 +146,12 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     // cluster and exchange their partial tiles through distributed shared memory
     g.cluster = allow_cluster && split_k >= 2 && split_k <= kDecMaxCluster && g.nchunks == g.ctas && g.mchunks == 1;
     const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
-    int st = (budget - 128 - decode_red_bytes(g.mb) - decode_xch_bytes(g.mb, g.cluster)) / decode_stage_bytes(g.mb);
+    const int xs = g.cluster ? split_k : 0;   // slices that meet in the exchange buffer
+    int st = (budget - 128 - decode_red_bytes(g.mb) - decode_xch_bytes(g.mb, xs)) / decode_stage_bytes(g.mb);
     if (st > kDecMaxStages) st = kDecMaxStages;
     if (st < 2) st = 2;
     g.stages = st;
-    g.smem_bytes = decode_smem_bytes(g.mb, st, g.cluster);
+    g.smem_bytes = decode_smem_bytes(g.mb, st, xs);
     return g;
 }
 
