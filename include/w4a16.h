@@ -118,7 +118,9 @@ int w4a16_dequant(const void *Wq, const void *S, const void *Z, uint16_t *W16,
  *   C   FP16 [M, N] row-major, fully overwritten (no beta)
  *   split_k   0 = automatic, else 1 <= split_k <= K/group (some paths cap it lower and
  *             return W4A16_ERR_SPLITK beyond their cap)
- * Results are bit-identical from run to run for fixed arguments.  If the chosen
+ * Results are bit-identical from run to run for fixed arguments (with split_k == 0 the schedule,
+ * and with it the order of the FP32 sums, is the library's choice for this entry point and device;
+ * it changes once, for good, if the device refuses a thread-block-cluster launch).  If the chosen
  * split needs workspace and too little is registered: W4A16_ERR_WORKSPACE.
  * Ordering: A, C and the workspace are touched in stream order.  The packed buffers Wq, S, Z
  * may be read (prefetched) while the previous kernel of the stream is still running, so
