@@ -59,6 +59,40 @@ def test_choose_split_k_is_always_acceptable(lib):
     assert lib.w4a16_workspace_bytes(4, 4096, 4096, 128, 4) >= 4 * 4 * 4096 * 4
 
 
+def test_path_and_schedule_rules_at_the_benchmark_shapes(lib):
+    """Host logic only (148 SMs assumed without a device, which is also what a B200 reports): the
+    path and the split the library reports for a shape are the ones it runs (w4a16_gemm asks the same
+    functions).  Values are the measured optima recorded beside the rules in the sources."""
+    DECODE, TILE = 2, 3
+    path = lambda M, N, K: lib.w4a16_choose_path(M, N, K, 128)
+    split = lambda M, N, K: lib.w4a16_choose_split_k(M, N, K, 128)
+    # up to 8 rows: always the warp-MMA kernel
+    for N, K in [(4096, 4096), (4096, 11008), (8192, 28672), (22016, 4096), (1536, 6144)]:
+        for M in (1, 4, 8):
+            assert path(M, N, K) == DECODE
+    # 9 .. 16 rows: the warp-MMA kernel where its K slices form clusters, else tcgen05
+    assert path(16, 4096, 11008) == DECODE and split(16, 4096, 11008) == 4
+    assert path(16, 4096, 4096) == DECODE
+    assert path(16, 12288, 4096) == TILE
+    assert path(16, 22016, 4096) == TILE
+    assert path(16, 8192, 28672) == TILE
+    # above 16 rows: tcgen05
+    for M in (17, 32, 64, 256, 4096):
+        assert path(M, 4096, 11008) == TILE
+    # slices per tile of the warp-MMA kernel: four (one cluster per tile) at config 2, whole tiles
+    # for the wide gate/up layer, at most six per cluster for narrow matrices
+    assert split(1, 4096, 11008) == 4
+    assert split(1, 4096, 4096) == 4
+    assert split(1, 22016, 4096) == 1
+    assert split(1, 12288, 4096) == 2
+    assert split(1, 1536, 6144) == 6
+    assert split(1, 2048, 8192) == 6
+    # wide batch tiles: whole tiles at M = 4096 (no partial tiles at all)
+    assert split(4096, 8192, 8192) == 1
+    # unsupported shapes are refused, not guessed
+    assert lib.w4a16_choose_path(1, 100, 4096, 128) < 0
+
+
 def test_argument_errors_are_reported_before_any_device_work(lib):
     buf = (ctypes.c_uint8 * 4096)()
     p = ctypes.addressof(buf)
