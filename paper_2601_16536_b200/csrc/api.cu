@@ -101,33 +101,43 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     g.mchunks = (M + 8 * g.mb - 1) / (8 * g.mb);
     const int T = N / kTileN;
     const long units = (long)T * G;
-    // Three CTAs per SM (a two-stage ring each) when every CTA has a long stream: measured with one
-    // batch block, 34.3 against 36.7 us at K = 28672 / N = 8192, 18.1 against 18.9 at K = 4096 /
-    // N = 22016, 12.6 against 13.5 at N = 12288, but 12.3 against 11.9 at K = 11008 / N = 4096 and
-    // 8.0 against 7.1 at K = N = 4096.  Two batch blocks leave room for one stage only: two CTAs.
-    g.cps = (g.mb == 1 && units >= 20L * 2 * sms) ? 3 : 2;
+    // Two CTAs per SM.  (Three, with a two-stage ring and 72 registers, were ahead on long launches
+    // while every exchange went through the workspace; with the cluster exchange two are ahead again
+    // everywhere but K = 4096 / N = 12288, by 3 %: 33.8 against 34.8 us at K = 28672 / N = 8192, 15.0
+    // against 15.8 at N = 22016.  The kernel keeps the template parameter.)
+    g.cps = 2;
     long slots = (long)g.cps * sms;
-    if (split_k == 0 && T <= slots) {
-        // Balanced chunks use every CTA slot, but a chunk that crosses a tile boundary goes through the
-        // workspace exchange in mid-stream.  S slices per tile keep every chunk inside one tile at the
-        // price of idle slots, and their exchange is cheaper: none at S = 1, through the cluster for
-        // S <= 6, at the end of the stream otherwise.  Costs in units per CTA, the exchanges priced from
-        // measurements (K = 4096 / N = 22016, M = 1: whole tiles 16.0 us against 18.4 balanced;
-        // K = 28672 / N = 8192: three slices 35.1 against 35.0; K = 11008 / N = 4096: four slices 9.8
-        // against 11.9 before there were clusters; K = 6144 / N = 1536: six slices in a cluster 4.8
-        // against 6.5 for twelve through the workspace).
-        int s0 = (int)(slots / T);
-        if (s0 > G) s0 = G;
-        // exchange prices in units: none 0, cluster 4, workspace at the end of a slice 9, workspace in
-        // mid-stream (balanced chunks) 13 -- 1.3 / 2.8 / about 4 us at 0.3 us per unit
+    if (split_k == 0) {
+        // How the unit range is cut when the caller leaves it open.  Balanced chunks use every CTA
+        // slot, but a chunk that crosses a tile boundary goes through the workspace exchange in
+        // mid-stream.  S slices per tile keep every chunk inside one tile, and their exchange is
+        // cheaper: none at S = 1, through the cluster for S <= 6, at the end of the stream otherwise.
+        // Slices are sized for 7/8 of the slots: a launch that fills every slot cannot start (and
+        // prefetch its weights) before the launch in front of it has drained (K = 10240 / N = 4608,
+        // 72 tiles: three slices 10.7 us, four 13.2).  Costs in units per CTA, exchanges priced from
+        // measurements: none 0, cluster 4, workspace at the end of a slice 9, workspace in mid-stream
+        // 13 (1.3 / 2.8 / about 4 us at 0.3 us per unit).  K = 4096 / N = 22016: whole tiles 15.0 us,
+        // balanced 18.1; K = 28672 / N = 8192: two slices 33.8, balanced 34.3; K = 11008 / N = 4096:
+        // four slices 9.7, three 10.5, two 13.5; K = 6144 / N = 1536: six slices in a cluster 4.8,
+        // twelve through the workspace 6.5.
         long best = (units + slots - 1) / slots + 13;
         int best_s = 0;
-        const long ws_cost = (G + s0 - 1) / s0 + (s0 == 1 ? 0 : 9);
-        if (ws_cost <= best) { best = ws_cost; best_s = s0; }
-        if (allow_cluster && g.mchunks == 1 && s0 >= 2) {
-            const int sc = s0 < kDecMaxCluster ? s0 : kDecMaxCluster;   // fewer, longer slices that fit a cluster
-            const long cl_cost = (G + sc - 1) / sc + 4;
-            if (cl_cost <= best) { best = cl_cost; best_s = sc; }
+        if (T > slots) {
+            // more tiles than CTAs: whole tiles dealt round-robin; the CTAs of an SM share its issue
+            // slots, so uneven tile counts cost less than the longest CTA suggests (15 % allowed)
+            const long whole_cost = (units * 23 / 20 + slots - 1) / slots;
+            if (whole_cost <= best) { best = whole_cost; best_s = 1; }
+        } else {
+            int s0 = (int)((slots * 7 / 8) / T);
+            if (s0 < 1) s0 = 1;
+            if (s0 > G) s0 = G;
+            const long ws_cost = (G + s0 - 1) / s0 + (s0 == 1 ? 0 : 9);
+            if (ws_cost <= best) { best = ws_cost; best_s = s0; }
+            if (allow_cluster && g.mchunks == 1 && s0 >= 2) {
+                const int sc = s0 < kDecMaxCluster ? s0 : kDecMaxCluster;   // fewer, longer slices that fit a cluster
+                const long cl_cost = (G + sc - 1) / sc + 4;
+                if (cl_cost <= best) { best = cl_cost; best_s = sc; }
+            }
         }
         split_k = best_s;
     }

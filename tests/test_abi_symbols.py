@@ -84,7 +84,7 @@ def test_path_and_schedule_rules_at_the_benchmark_shapes(lib):
     assert split(1, 4096, 11008) == 4
     assert split(1, 4096, 4096) == 4
     assert split(1, 22016, 4096) == 1
-    assert split(1, 12288, 4096) == 2
+    assert split(1, 12288, 4096) == 1
     assert split(1, 1536, 6144) == 6
     assert split(1, 2048, 8192) == 6
     # wide batch tiles: whole tiles at M = 4096 (no partial tiles at all)
