@@ -226,7 +226,8 @@ TileGeom tile_geom(int M, int N, int G, int split_k, int sms, int max_smem) {
         // waves (tiles > SMs) avoid that at the price of idle SMs.  Cost model in groups per CTA; the
         // constants are fitted to measurements (K = 11008 / N = 4096, K = 28672 / N = 8192 and
         // K = N = 8192 with M up to 4096).
-        const long penalty = 6 + g.mt / 8;
+        // (narrow tiles: K = 4096 / N = 12288, M = 16: 96 whole tiles 13.8 us, balanced chunks 16.3)
+        const long penalty = (g.mt <= 32 ? 10 : 6) + g.mt / 8;
         const long balanced_cost = (g.tiles * G + sms - 1) / sms + penalty;
         int s0 = 1;
         long classic_cost;
