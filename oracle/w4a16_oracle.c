@@ -9,9 +9,9 @@
  *
  * Conventions (the paper leaves them open; these are the readings used):
  *   - W is unsigned INT4, 0..15, with an integer zero point z in 0..15.
- *   - INT4 values are stored 8 per 32-bit word along K ("packed into larger
- *     data types such as INT32", Section 2.2): word Wq[kk, n] of the row-major
- *     array [K/8, N] holds q[8*kk + i, n] in bits 4i .. 4i+3.
+ *   - INT4 values are stored 8 per 32-bit word along K (storage packing,
+ *     Section 2.2): word Wq[kk, n] of the row-major array [K/8, N] holds
+ *     q[8*kk + i, n] in bits 4i .. 4i+3.
  *   - s and z are per (group, column): S f16 [K/group, N], Z u8 [K/group, N].
  *   - "Dequantize to FP16" (Algorithm 1, Phase 1): the multiplicand is the
  *     FP16-rounded weight  w16 = fp16_rn((q - z) * s).  (q - z) is exact and
