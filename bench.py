@@ -7,9 +7,13 @@ the packed weights so that every call streams its weights from HBM (the copies t
 than 512 MB; B200's L2 is 126 MB).  The metric is effective HBM bandwidth = algorithmic
 bytes (packed weights + FP16 scales + 4-bit zeros + activations + output) / time.
 
-Prints ONE JSON line (see the keys below).  `--impl reference` times the CPU oracle on the
-host cores instead.  Under torchrun each rank runs an independent replica (the path has no
-exchange step) and rank 0 reports the aggregate.
+The LAST line of stdout is one compact JSON object (the headline: value, roofline, e2e,
+cpu_baseline, clocks ...; under 4 KB).  The bulky per-case table (every case of every config,
+explicit split_k sweep, warm-L2 times, FP16 x FP16 reference) is written to
+--cases-file and echoed on earlier stdout lines prefixed "CASE ".  `--impl reference` times the
+CPU oracle on the host cores instead.  Under torchrun each rank runs an independent replica (the
+path has no exchange step) and rank 0 reports the aggregate; `--gpus N` without torchrun starts
+the N ranks itself.
 """
 from __future__ import annotations
 
@@ -210,22 +214,70 @@ def _capture(fn, n, torch):
     return g
 
 
-def _time_calls(fn, n_warm, n_timed, torch, per_graph=32):
-    """Seconds per call: `fn` captured per_graph times into a CUDA graph, replayed."""
+def _replay_times(graph, reps, torch):
+    """Device seconds of each of `reps` replays of one graph (CUDA events on the launching stream)."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    ev[0].record()
+    for r in range(reps):
+        graph.replay()
+        ev[r + 1].record()
+    torch.cuda.synchronize()
+    return [ev[r].elapsed_time(ev[r + 1]) * 1e-3 for r in range(reps)]
+
+
+def _time_calls(fn, n_warm, n_timed, torch, per_graph=32, reps=5):
+    """Seconds per call of `fn` inside replayed CUDA graphs of `per_graph` calls: (median, min) over
+    at least `reps` replays (and at least n_timed calls in total)."""
     for _ in range(max(3, n_warm)):
         fn()
     torch.cuda.synchronize()
     g = _capture(fn, per_graph, torch)
-    reps = max(1, n_timed // per_graph)
     g.replay()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        g.replay()
-    e1.record()
-    torch.cuda.synchronize()
-    return e0.elapsed_time(e1) * 1e-3 / (reps * per_graph)
+    reps = max(reps, -(-n_timed // per_graph))
+    t = [x / per_graph for x in _replay_times(g, reps, torch)]
+    return statistics.median(t), min(t)
+
+
+def summary_line(d):
+    """The compact last line: the headline object serialised without the per-case table."""
+    return json.dumps(d, separators=(",", ":"))
+
+
+def emit(summary, cases, cases_file, out=None):
+    """Write the per-case table to `cases_file` (if it can be written) and as "CASE {...}" lines, then
+    the compact summary as the LAST line of `out`."""
+    out = out or sys.stdout
+    if cases_file:
+        try:
+            os.makedirs(os.path.dirname(os.path.abspath(cases_file)), exist_ok=True)
+            with open(cases_file, "w") as f:
+                json.dump({"summary": summary, "cases": cases}, f, indent=1)
+            summary = dict(summary, cases_file=os.path.relpath(cases_file, ROOT))
+        except OSError:
+            pass
+    for c in cases:
+        out.write("CASE " + json.dumps(c, separators=(",", ":")) + "\n")
+    out.write(summary_line(summary) + "\n")
+    out.flush()
+
+
+def _r(x, nd=4):
+    return None if x is None else round(float(x), nd)
+
+
+def _case_record(c_config, layer, M, K, N, sec_med, sec_min, path, peaks, wl):
+    hbm_peak, tc_peak = peaks
+    byts = wl.algorithmic_bytes(M, K, N)
+    fl = 2.0 * M * N * K
+    t_hbm, t_tc = byts / (hbm_peak * 1e9), fl / (tc_peak * 1e12)
+    return {"config": c_config, "layer": layer, "M": M, "K": K, "N": N, "path": path,
+            "us": _r(sec_med * 1e6, 3), "us_min": _r(sec_min * 1e6, 3),
+            "eff_GBps": _r(byts / sec_med / 1e9, 1), "tflops": _r(fl / sec_med / 1e12, 2),
+            "bound": "tensor" if t_tc > t_hbm else "hbm",
+            "roofline_frac": _r(max(t_hbm, t_tc) / sec_med),
+            # the same against the nominal peaks (8 TB/s, 2250 TFLOP/s dense FP16)
+            "roofline_frac_nominal": _r(max(byts / 8e12, fl / 2250e12) / sec_med)}
 
 
 def run_ours(args):
@@ -244,6 +296,7 @@ def run_ours(args):
     from paper_2601_16536_b200 import workloads as wl
     B.load()
     hbm_peak, tc_peak, peak_kind = _peaks()
+    peaks = (hbm_peak, tc_peak)
 
     K, N = SWEEP_K, SWEEP_N
     layer = Layer(K, N, 2000, torch, B, wl)
@@ -251,20 +304,18 @@ def run_ours(args):
     acts = [_to_dev(a, torch) for a in acts_np]
     outs = [torch.empty((M, N), dtype=torch.float16, device="cuda") for M in SWEEP_M]
     splits = [args.split_k for M in SWEEP_M]   # 0 = the library's own schedule
-    ws_need = max([B.w4a16_workspace_bytes(M, N, K, 128, s) for M, s in zip(SWEEP_M, splits)] + [16384])
+    ws_need = max([B.w4a16_workspace_bytes(M, N, K, 128, s) for M in SWEEP_M for s in (0, 1, 2, 4, 8, 16)]
+                  + [16384])
     extra_cases = []
-    if args.configs:
-        for c in wl.CASES:
-            if c.config in args.configs and not (c.config == 2):
-                if world > 1 and c.config != 2:
-                    continue        # the per-case table is a 1-GPU report
-                extra_cases.append(c)
+    if args.configs and world == 1:          # the per-case table is a 1-GPU report
+        extra_cases = [c for c in wl.CASES if c.config in args.configs and c.config != 2]
         # the tensor-bound config 5 goes last: right after its long launches (and their FP16 references)
-        # the GPU runs the next short launches 30-40 % slower for a while (power state), which used to
-        # land on whichever small layer came next
+        # the GPU runs the next short launches 30-40 % slower for a while (power state)
         extra_cases.sort(key=lambda c: c.config == 5)
         for c in extra_cases:
-            ws_need = max(ws_need, B.w4a16_workspace_bytes(c.M, c.N, c.K, 128, 0))
+            for s in (0, 2, 4, 8, 16):
+                if s <= c.K // 128:
+                    ws_need = max(ws_need, B.w4a16_workspace_bytes(c.M, c.N, c.K, 128, s))
     ws = B.ensure_workspace(ws_need)
 
     def step():
@@ -274,119 +325,135 @@ def run_ours(args):
     launches_per_step = len(SWEEP_M)   # one kernel per GEMM: the Split-K reduce is inside it
     step_bytes = sum(wl.algorithmic_bytes(M, K, N) for M in SWEEP_M)
 
-    # ---- main timed region: W warm-up steps, exactly K steps, device events, max over ranks.
-    # The steps are captured into CUDA graphs (one rotation through the weight copies each) and
-    # replayed, so the timed region holds exactly steps x 5 kernel launches and no host work.
+    # ---- main timed region.  W warm-up steps; then the region of exactly `steps` steps is captured
+    # into a CUDA graph (no host work inside) and replayed `reps` times, each replay bracketed by
+    # CUDA events on the launching stream.  ms_per_step is the median replay (the minimum is reported
+    # beside it); reps is sized so that the timed work is at least ~0.15 s whatever --steps is.
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
-    chunk = max(1, min(args.steps, layer.copies))
-    g_main = _capture(step, chunk, torch)
-    reps, rem = divmod(args.steps, chunk)
-    g_rem = _capture(step, rem, torch) if rem else None
+    g_main = _capture(step, args.steps, torch)
     g_main.replay()
     torch.cuda.synchronize()
+    probe = _replay_times(g_main, 2, torch)[-1]
+    reps = max(20, min(2000, int(0.15 / max(probe, 1e-6)) + 1))
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if not args.no_clocks:
         sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        g_main.replay()
-    if g_rem is not None:
-        g_rem.replay()
-    e1.record()
-    torch.cuda.synchronize()
+    rep_times = _replay_times(g_main, reps, torch)
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
-    elapsed = e0.elapsed_time(e1) * 1e-3
+    timed_total = sum(rep_times)
     if not args.no_clocks:
         # keep the same load running until the sampler has seen ~0.6 s of it
-        t_end = time.perf_counter() + max(0.0, 0.6 - elapsed)
+        t_end = time.perf_counter() + max(0.0, 0.6 - timed_total)
         while time.perf_counter() < t_end:
             g_main.replay()
             torch.cuda.synchronize()
     clocks = sampler.stop()
-    elapsed = max_over_ranks(elapsed, dist, "cuda")
+    elapsed = max_over_ranks(statistics.median(rep_times), dist, "cuda")     # one region of `steps` steps
+    elapsed_min = max_over_ranks(min(rep_times), dist, "cuda")
     assert B.w4a16_device_status() == 0, "a kernel reported a device-side timeout"
     value = whole_job_value(step_bytes, args.steps, world, elapsed)
 
-    # ---- per-case numbers (each M alone, same rotation)
+    # ---- per-case numbers (each M alone, same rotation, same launch form)
     cases = []
     per_call = {}
+    extras_error = None
+    sweep_splits = (1, 2, 4, 8, 16)
+
+    def split_sweep(rec, A, lay, C, M, Kc, Nc, calls):
+        """Explicit split_k beside the library's own schedule (the paper takes S as an input)."""
+        best_s, best = None, None
+        rec["us_by_split_k"] = {}
+        for s in sweep_splits:
+            if s > Kc // 128:
+                continue
+            try:
+                sec, _ = _time_calls(lambda: B.w4a16_gemm(A, lay.take(), C, split_k=s), 5, calls, torch)
+            except B.W4A16Error:
+                continue
+            rec["us_by_split_k"][str(s)] = _r(sec * 1e6, 3)
+            if best is None or sec < best:
+                best_s, best = s, sec
+        rec["us_split_k_1"] = rec["us_by_split_k"].get("1")
+        rec["best_explicit_split_k"] = best_s
+        rec["auto_vs_best_explicit"] = _r(rec["us"] / (best * 1e6), 3) if best else None
+
     for i, M in enumerate(SWEEP_M):
-        sec = _time_calls(lambda: B.w4a16_gemm(acts[i], layer.take(), outs[i], split_k=splits[i]),
-                          20, args.case_calls, torch)
-        byts = wl.algorithmic_bytes(M, K, N)
-        per_call[M] = sec
-        cases.append({"config": 2, "layer": "down_proj", "M": M, "K": K, "N": N, "split_k": splits[i],
-                      "path": PATH_NAMES.get(B.w4a16_choose_path(M, N, K), "?"),
-                      "us": sec * 1e6, "eff_GBps": byts / sec / 1e9, "tflops": 2.0 * M * N * K / sec / 1e12,
-                      "roofline_frac": max(byts / (hbm_peak * 1e9), 2.0 * M * N * K / (tc_peak * 1e12)) / sec})
-    # split_k = 1 ("data parallel" in the paper's comparison) beside the chosen split
-    for i, M in enumerate(SWEEP_M):
-        sec = _time_calls(lambda: B.w4a16_gemm(acts[i], layer.take(), outs[i], split_k=1), 10,
-                          max(50, args.case_calls // 4), torch)
-        cases[i]["us_split_k_1"] = sec * 1e6
+        med, mn = _time_calls(lambda: B.w4a16_gemm(acts[i], layer.take(), outs[i], split_k=splits[i]),
+                              20, args.case_calls, torch)
+        per_call[M] = med
+        rec = _case_record(2, "down_proj", M, K, N, med, mn, PATH_NAMES.get(B.w4a16_choose_path(M, N, K), "?"),
+                           peaks, wl)
+        rec["split_k"] = splits[i]
+        rec["chosen_split_k"] = B.w4a16_choose_split_k(M, N, K)
+        cases.append(rec)
+    try:
+        if rank == 0 and world == 1 and not args.headline_only:
+            for i, M in enumerate(SWEEP_M):
+                split_sweep(cases[i], acts[i], layer, outs[i], M, K, N, max(64, args.case_calls // 4))
+                # warm L2: the same packed copy every call (23 MB stay in the 126 MB L2) -- labelled, not the metric
+                sec, _ = _time_calls(lambda: B.w4a16_gemm(acts[i], layer.packed[0], outs[i], split_k=splits[i]),
+                                     5, max(64, args.case_calls // 4), torch)
+                cases[i]["us_warm_l2"] = _r(sec * 1e6, 3)
 
-    # cuBLAS / PyTorch FP16 x FP16 on pre-dequantized weights: a reference point, not our path
-    if not args.no_cublas:
-        w16 = [B.w4a16_dequant(layer.packed[0]).clone() for _ in range(6)]
-        idx = [0]
+            # cuBLAS / PyTorch FP16 x FP16 on pre-dequantized weights: a reference point, not our path
+            if not args.no_cublas:
+                w16 = [B.w4a16_dequant(layer.packed[0]).clone() for _ in range(6)]
+                idx = [0]
 
-        def mm(i):
-            torch.matmul(acts[i], w16[idx[0] % len(w16)], out=outs[i])
-            idx[0] += 1
-        for i, M in enumerate(SWEEP_M):
-            sec = _time_calls(lambda: mm(i), 10, max(50, args.case_calls // 4), torch)
-            cases[i]["torch_fp16_matmul_us"] = sec * 1e6
-            cases[i]["speedup_vs_fp16"] = sec / per_call[M]
-        del w16
+                def mm(i):
+                    torch.matmul(acts[i], w16[idx[0] % len(w16)], out=outs[i])
+                    idx[0] += 1
+                for i, M in enumerate(SWEEP_M):
+                    sec, _ = _time_calls(lambda: mm(i), 10, max(50, args.case_calls // 4), torch)
+                    cases[i]["torch_fp16_matmul_us"] = _r(sec * 1e6, 3)
+                    cases[i]["speedup_vs_fp16"] = _r(sec / per_call[M], 3)
+                del w16
 
-    # other configs on request (each case alone, rotating copies)
-    cur = None
-    cur_w16 = None
-    for c in extra_cases:
-        if cur is None or (cur.K, cur.N) != (c.K, c.N):
+            # other configs (each case alone, rotating copies)
             cur = None
             cur_w16 = None
-            torch.cuda.empty_cache()
-            cur = Layer(c.K, c.N, c.seed, torch, B, wl)
-        A = _to_dev(wl.draw_activations(c.M, c.K, c.seed, c.a_sigma, c.outliers), torch)
-        C = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
-        s = 0
-        sec = _time_calls(lambda: B.w4a16_gemm(A, cur.take(), C, split_k=s), 10,
-                          max(20, args.case_calls // 4), torch)
-        byts = wl.algorithmic_bytes(c.M, c.K, c.N)
-        fl = 2.0 * c.M * c.N * c.K
-        rec = {"config": c.config, "layer": c.name, "M": c.M, "K": c.K, "N": c.N, "split_k": s,
-               "path": PATH_NAMES.get(B.w4a16_choose_path(c.M, c.N, c.K), "?"),
-               "us": sec * 1e6, "eff_GBps": byts / sec / 1e9, "tflops": fl / sec / 1e12,
-               "bound": "tensor" if fl / (tc_peak * 1e12) > byts / (hbm_peak * 1e9) else "hbm",
-               "roofline_frac": max(byts / (hbm_peak * 1e9), fl / (tc_peak * 1e12)) / sec}
-        if c.config == 6:
-            # the paper's Figure 2 comparison: one slice ("data parallel") beside the chosen schedule
-            sec1 = _time_calls(lambda: B.w4a16_gemm(A, cur.take(), C, split_k=1), 5,
-                               max(20, args.case_calls // 8), torch)
-            rec["us_split_k_1"] = sec1 * 1e6
-            rec["splitk_speedup"] = sec1 / sec
-        if not args.no_cublas:
-            if cur_w16 is None:
-                ncopy = max(2, min(6, (MIN_ROTATION_BYTES // 2) // (c.K * c.N * 2) + 1))
-                cur_w16 = [B.w4a16_dequant(cur.packed[0]).clone() for _ in range(ncopy)]
-            k16 = [0]
+            for c in extra_cases:
+                if cur is None or (cur.K, cur.N) != (c.K, c.N):
+                    cur = None
+                    cur_w16 = None
+                    torch.cuda.empty_cache()
+                    cur = Layer(c.K, c.N, c.seed, torch, B, wl)
+                A = _to_dev(wl.draw_activations(c.M, c.K, c.seed, c.a_sigma, c.outliers), torch)
+                C = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
+                med, mn = _time_calls(lambda: B.w4a16_gemm(A, cur.take(), C, split_k=0), 10,
+                                      max(20, args.case_calls // 4), torch)
+                rec = _case_record(c.config, c.name, c.M, c.K, c.N, med, mn,
+                                   PATH_NAMES.get(B.w4a16_choose_path(c.M, c.N, c.K), "?"), peaks, wl)
+                rec["split_k"] = 0
+                rec["chosen_split_k"] = B.w4a16_choose_split_k(c.M, c.N, c.K)
+                if c.config in (3, 6):
+                    split_sweep(rec, A, cur, C, c.M, c.K, c.N, max(20, args.case_calls // 8))
+                    if rec.get("us_split_k_1"):
+                        rec["splitk_speedup"] = _r(rec["us_split_k_1"] / rec["us"], 3)
+                if not args.no_cublas:
+                    if cur_w16 is None:
+                        ncopy = max(2, min(6, (MIN_ROTATION_BYTES // 2) // (c.K * c.N * 2) + 1))
+                        cur_w16 = [B.w4a16_dequant(cur.packed[0]).clone() for _ in range(ncopy)]
+                    k16 = [0]
 
-            def mm16():
-                torch.matmul(A, cur_w16[k16[0] % len(cur_w16)], out=C)
-                k16[0] += 1
-            sec16 = _time_calls(mm16, 5, max(20, args.case_calls // 8), torch, per_graph=8)
-            rec["torch_fp16_matmul_us"] = sec16 * 1e6
-            rec["speedup_vs_fp16"] = sec16 / sec
-        cases.append(rec)
+                    def mm16():
+                        torch.matmul(A, cur_w16[k16[0] % len(cur_w16)], out=C)
+                        k16[0] += 1
+                    sec16, _ = _time_calls(mm16, 5, max(20, args.case_calls // 8), torch, per_graph=8)
+                    rec["torch_fp16_matmul_us"] = _r(sec16 * 1e6, 3)
+                    rec["speedup_vs_fp16"] = _r(sec16 / med, 3)
+                cases.append(rec)
+            cur = None
+            cur_w16 = None
+    except Exception as exc:   # the headline below does not depend on the optional table
+        extras_error = "%s: %s" % (type(exc).__name__, exc)
 
     # ---- end to end through the host-buffer entry point (H2D of A and D2H of C inside the region)
     hA = [torch.from_numpy(a.view(np.float16)).pin_memory() for a in acts_np]
@@ -399,33 +466,46 @@ def run_ours(args):
     for _ in range(max(3, args.warmup)):
         step_e2e()
     torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        step_e2e()
-    torch.cuda.synchronize()
-    e2e_elapsed = time.perf_counter() - t0
-    e2e_elapsed = max_over_ranks(e2e_elapsed, dist, "cuda")
-    e2e_value = whole_job_value(step_bytes, args.steps, world, e2e_elapsed)
+    e2e_steps = max(args.steps, 200)      # long enough to time on the wall clock
+    e2e_times = []
+    for _ in range(5):
+        if dist:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_e2e()
+        torch.cuda.synchronize()
+        e2e_times.append(time.perf_counter() - t0)
+    e2e_elapsed = max_over_ranks(statistics.median(e2e_times), dist, "cuda")
+    e2e_value = whole_job_value(step_bytes, e2e_steps, world, e2e_elapsed)
 
-    # ---- roofline of the dominant kernel (the decode GEMM kernel at M = 16, the heaviest call)
-    dom_M = SWEEP_M[-1]
-    dom_bytes = wl.algorithmic_bytes(dom_M, K, N)
-    achieved = dom_bytes / per_call[dom_M] / 1e9
-    dom_kernel = PATH_NAMES.get(B.w4a16_choose_path(dom_M, N, K), "?")
-    roofline = {"bound": "hbm", "kernel": dom_kernel, "case": "M=%d K=%d N=%d" % (dom_M, K, N),
-                "achieved": achieved, "peak": hbm_peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES.get(dom_kernel),
-                "algorithmic_bytes_per_launch": dom_bytes,
-                "launch_us": per_call[dom_M] * 1e6,
-                "sweep_frac": value / world / hbm_peak}
+    # ---- roofline of the dominant kernel.  Every launch of the timed region is gemm_decode_kernel (one
+    # per GEMM), so its average launch duration over the region is region time / launches, and the
+    # algorithmic bytes of an average launch are step bytes / launches per step.
+    dom_kernel = PATH_NAMES.get(B.w4a16_choose_path(SWEEP_M[0], N, K), "?")
+    launch_us = elapsed / (args.steps * launches_per_step) * 1e6
+    bytes_per_launch = step_bytes / launches_per_step
+    achieved = bytes_per_launch / launch_us / 1e3
+    heavy = SWEEP_M[-1]
+    roofline = {"bound": "hbm", "kernel": dom_kernel,
+                "launches": "the %d launches of a step (M = %s), averaged over the timed region"
+                            % (launches_per_step, "/".join(str(m) for m in SWEEP_M)),
+                "achieved": _r(achieved, 1), "peak": hbm_peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
+                "frac": _r(achieved / hbm_peak), "frac_of_nominal_8TBps": _r(achieved / 8000.0),
+                "traffic": NCU_TRAFFIC_BYTES.get(dom_kernel),
+                "algorithmic_bytes_per_launch": int(bytes_per_launch), "launch_us": _r(launch_us, 3),
+                "launch_us_by_M": {str(M): _r(per_call[M] * 1e6, 3) for M in SWEEP_M},
+                "frac_by_M": {str(M): _r(wl.algorithmic_bytes(M, K, N) / per_call[M] / 1e9 / hbm_peak)
+                              for M in SWEEP_M},
+                "heaviest_launch": "M=%d: %s" % (heavy, PATH_NAMES.get(B.w4a16_choose_path(heavy, N, K), "?"))}
 
-    # ---- CPU baseline: the oracle on the full sweep once (rank 0, N = 1 only)
+    # ---- CPU baseline: the oracle on whole steps (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         worst, reps_cpu, dt = 0.0, 0, 0.0
+        step()
+        torch.cuda.synchronize()
         while dt < 10.0 and reps_cpu < 64:     # whole steps until about 10 s of CPU work
             t0 = time.perf_counter()
             refs = [oracle.gemm(acts_np[i], layer.raw["Wq"], layer.raw["S"], layer.raw["Z"], M, N, K, 128)
@@ -433,60 +513,64 @@ def run_ours(args):
             dt += time.perf_counter() - t0
             reps_cpu += 1
         for i, M in enumerate(SWEEP_M):
-            got = outs[i].cpu().numpy().astype(np.float64)   # result of the last timed call
+            got = outs[i].cpu().numpy().astype(np.float64)   # result of the last call
             worst = max(worst, float(np.max(np.abs(got - refs[i]) / (1.0 + np.abs(refs[i])))))
-        cpu = {"value": step_bytes * reps_cpu / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(),
+        cpu = {"value": _r(step_bytes * reps_cpu / dt / 1e9, 5), "unit": UNIT, "cores": oracle.num_threads(),
                "kind": "oracle",
                "sample": "%d full steps (all 5 GEMMs, all columns), %.1f s of CPU time" % (reps_cpu, dt),
-               "max_elem_err_vs_gpu": worst}
+               "max_elem_err_vs_gpu": _r(worst, 6)}
 
     # the tensor-bound end of the path: the largest prefill case that was timed (config 5)
     roofline_tensor = None
     big = [c for c in cases if c["config"] == 5]
     if big:
         b = max(big, key=lambda c: c["M"])
-        peaks = {}
+        pk = {}
         try:
-            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+            pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
         except Exception:
             pass
-        sustained = float(peaks.get("bf16_tflops_sustained", 1400.0))
+        sustained = float(pk.get("bf16_tflops_sustained", 1400.0))
         roofline_tensor = {"bound": "tensor", "kernel": b["path"], "case": "M=%d K=%d N=%d" % (b["M"], b["K"], b["N"]),
-                           "achieved": b["tflops"], "peak": tc_peak, "peak_kind": "of " + peak_kind +
-                           " (burst; FP16 takes the BF16 figure, same nominal rate)", "unit": "TFLOP/s",
-                           "frac": b["tflops"] / tc_peak, "frac_of_sustained_peak": b["tflops"] / sustained,
+                           "achieved": b["tflops"], "peak": tc_peak,
+                           "peak_kind": "of " + peak_kind + " (burst; FP16 takes the BF16 figure, same nominal rate)",
+                           "unit": "TFLOP/s", "frac": _r(b["tflops"] / tc_peak),
+                           "frac_of_sustained_peak": _r(b["tflops"] / sustained),
+                           "frac_of_nominal_2250": _r(b["tflops"] / 2250.0),
                            "launch_us": b["us"], "traffic": NCU_TRAFFIC_BYTES_TILE}
     # config 4: the four layers of one transformer block, summed per batch size
     block_sums = {}
     for c in cases:
         if c["config"] == 4:
-            block_sums.setdefault(c["M"], 0.0)
-            block_sums[c["M"]] += c["us"]
+            block_sums[str(c["M"])] = _r(block_sums.get(str(c["M"]), 0.0) + c["us"], 2)
 
     if rank == 0:
-        print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": elapsed / args.steps * 1e3, "higher_is_better": True,
+        summary = {
+            "metric": METRIC, "value": _r(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": _r(elapsed / args.steps * 1e3, 6),
+            "ms_per_step_min": _r(elapsed_min / args.steps * 1e3, 6), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "group": 128, "accumulate": "f32", "split_k": splits,
+            "config": {"workload": WORKLOAD, "group": 128, "accumulate": "f32", "split_k": splits[0],
                        "l2": "cold: %d packed weight copies (%d MB) rotated, every call reads HBM"
                              % (layer.copies, layer.copies * (K * N // 2) >> 20),
-                       "launch": "CUDA graphs of %d steps, replayed" % chunk,
-                       "multi_gpu": "replicas only"},
+                       "launch": "one CUDA graph of the %d steps, replayed %d times; ms_per_step = median replay"
+                                 % (args.steps, reps),
+                       "timed_s": _r(timed_total, 4), "multi_gpu": "replicas only"},
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT,
+            "e2e": {"value": _r(e2e_value, 2), "unit": UNIT,
                     "h2d_bytes_per_step": sum(2 * M * K for M in SWEEP_M),
                     "d2h_bytes_per_step": sum(2 * M * N for M in SWEEP_M),
-                    "ms_per_step": e2e_elapsed / args.steps * 1e3,
-                    "note": "activations from pinned host memory, result to pinned host memory; "
-                            "packed weights resident in HBM"},
-            "gpu_launches": launches_per_step * args.steps,
+                    "ms_per_step": _r(e2e_elapsed / e2e_steps * 1e3, 6), "steps": e2e_steps,
+                    "note": "A from pinned host memory, C to pinned host memory, weights resident; wall clock"},
+            "gpu_launches": launches_per_step * args.steps * reps,
             "roofline": roofline,
             "roofline_tensor": roofline_tensor,
             "config4_block_us_by_M": block_sums,
             "cpu_baseline": cpu,
-            "cases": cases,
-        }))
+        }
+        if extras_error:
+            summary["cases_error"] = extras_error[:200]
+        emit(summary, cases, args.cases_file)
     del ws
     if dist:
         dist.destroy_process_group()
@@ -522,7 +606,7 @@ def run_one(args):
     if args.graph:
         # the same call inside replayed CUDA graphs: device time of back-to-back launches
         g_us = _time_calls(lambda: B.w4a16_gemm(A, layer.take(), C, split_k=args.split_k, path=args.path),
-                           3, max(args.calls, 64), torch, per_graph=min(32, max(2, layer.copies))) * 1e6
+                           3, max(args.calls, 64), torch, per_graph=min(32, max(2, layer.copies)))[0] * 1e6
         hbm_peak, tc_peak, _ = _peaks()
         out.update(us_per_call_graph=g_us, eff_GBps=byts / g_us / 1e3, tflops=2.0 * M * N * K / g_us / 1e6,
                    roofline_frac=max(byts / (hbm_peak * 1e3), 2.0 * M * N * K / (tc_peak * 1e6)) / g_us)
@@ -549,16 +633,34 @@ def main():
     ap.add_argument("--graph", action="store_true", help="--one: also time the call inside CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="kernel path of --one (0 auto, 1 simple, 2 decode, 3 tile)")
     ap.add_argument("--rotation-mb", type=int, default=512, help="bytes of rotating weight copies of --one")
+    ap.add_argument("--cases-file", default=os.path.join(ROOT, "gpurun_out", "bench_cases.json"),
+                    help="where the per-case table goes ('' = nowhere)")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the per-case table (other configs, split_k sweep, FP16 reference)")
     args = ap.parse_args()
     if args.one:
         run_one(args)
         return
+    world_env = os.environ.get("WORLD_SIZE")
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
+    if world_env is None and args.gpus > 1:
+        # not under torchrun: start the N replicas ourselves (one process per GPU, rendezvous on 127.0.0.1)
+        import socket
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
+    if world_env is not None and int(world_env) != args.gpus:
+        raise SystemExit("--gpus %d but WORLD_SIZE=%s: launch one rank per GPU" % (args.gpus, world_env))
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args)
     else:
-        args.steps = 2000 if args.steps is None else args.steps
+        args.steps = 100 if args.steps is None else args.steps
         args.warmup = max(3, 20 if args.warmup is None else args.warmup)
         run_ours(args)
 

@@ -21,8 +21,8 @@
  *   - Device code exists for sm_100a only; on any other device the launching calls
  *     return W4A16_ERR_ARCH.
  *
- * Raw layout (what w4a16_pack consumes; Section 2.2: "4-bit values must be packed into
- * larger data types such as INT32"):
+ * Raw layout (what w4a16_pack consumes; storage packing of 4-bit values into 32-bit words,
+ * Section 2.2):
  *   Wq_raw  uint32 [K/8, N] row-major; bits 4i..4i+3 of Wq_raw[kk, n] hold q[8 kk + i, n]
  *   S_raw   FP16   [K/group, N] row-major
  *   Z_raw   uint8  [K/group, N] row-major, one zero point (0..15) per byte
@@ -125,7 +125,9 @@ int w4a16_dequant(const void *Wq, const void *S, const void *Z, uint16_t *W16,
  * Ordering: A, C and the workspace are touched in stream order.  The packed buffers Wq, S, Z
  * may be read (prefetched) while the previous kernel of the stream is still running, so
  * they must not be written by in-flight work other than a w4a16_pack enqueued earlier on the
- * same device (the library orders the next GEMM launch after it); pack weights once, at load. */
+ * same stream (the library makes the first GEMM launch on each stream after a pack a fully
+ * ordered one; a pack on ANOTHER stream needs the caller's own event or synchronisation before
+ * the GEMM, as for any cross-stream dependency); pack weights once, at load. */
 int w4a16_gemm(const uint16_t *A, const void *Wq, const void *S, const void *Z, uint16_t *C,
                int M, int N, int K, int group, int split_k, w4a16_stream_t stream);
 
@@ -160,8 +162,9 @@ int w4a16_gemm_host(const uint16_t *A_host, uint16_t *A_dev, const void *Wq, con
  *     process exits, whether or not this call is ever made.
  *   - Limit: a shape / split_k whose scratch need (16 KiB of counters + the partial tiles, the
  *     same amount w4a16_workspace_bytes reports for the small-M kernel) exceeds the array is
- *     rejected with W4A16_ERR_WORKSPACE and nothing is launched.  Every M <= 16 with
- *     split_k = 0 fits; large explicit split_k on wide N may not.
+ *     rejected with W4A16_ERR_WORKSPACE and nothing is launched.  A schedule of whole tiles
+ *     (split_k = 1, or split_k = 0 where the library picks whole tiles) needs no scratch and
+ *     always fits; every M <= 16 with split_k = 0 fits; large explicit split_k on wide N may not.
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress with that device current) and sets a kernel attribute; make that
  *     first call outside any stream capture.  Later calls only enqueue work.
@@ -175,11 +178,25 @@ int w4a16_gemm_static_ws(const uint16_t *A, const void *Wq, const void *S, const
                          uint16_t *C, int M, int N, int K, int group, int split_k,
                          w4a16_stream_t stream);
 
-/* Kernels never wait without a limit: a wait that runs out records a code in a status
- * word on the device and the kernel returns.  This call synchronises the current
- * device, copies the word to *status_out (0 = no kernel ever gave up) and clears it.
- * Returns W4A16_ERR_DEVICE_STATUS if it was nonzero. */
+/* Every wait inside the kernels on a barrier or on another CTA has a limit (two seconds): a
+ * wait that runs out records a code in a status word on the device, the kernel releases what
+ * it holds and returns.  (The one instruction that can block without a limit is the tensor-
+ * memory allocation of the tile kernel; it cannot wait on another CTA of this library because
+ * the kernel asks for more than half of an SM's shared memory, so two of its CTAs never share
+ * an SM, and each frees its columns before it returns.)
+ * w4a16_device_status synchronises the current device, copies the word to *status_out
+ * (0 = no kernel gave up since the last call; bit 0 = a barrier wait ran out) and clears it.
+ * If it was nonzero the call also zeroes the ticket counters of the registered workspace (a
+ * kernel that gave up may have left them mid-count) and returns W4A16_ERR_DEVICE_STATUS; the
+ * output of the GEMM calls since the previous status check is then undefined, later calls
+ * work normally. */
 int w4a16_device_status(int *status_out);
+
+/* Diagnostic for the path above, no counterpart in the paper: enqueues a one-warp kernel whose
+ * only action is a bounded wait, limit `limit_us` microseconds (1 .. 100000), on a barrier that
+ * nothing ever arrives on.  The wait runs out, the kernel records the code and returns; the next
+ * w4a16_device_status reports it.  Nothing faults and the context stays usable. */
+int w4a16_selftest_wait_timeout(unsigned limit_us, w4a16_stream_t stream);
 
 #ifdef __cplusplus
 }

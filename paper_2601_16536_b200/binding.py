@@ -25,7 +25,7 @@ EXPORTS = (
     "w4a16_strerror", "w4a16_packed_wq_bytes", "w4a16_packed_s_bytes", "w4a16_packed_z_bytes",
     "w4a16_workspace_bytes", "w4a16_set_workspace", "w4a16_choose_split_k",
     "w4a16_choose_split_k_ex", "w4a16_choose_path", "w4a16_pack", "w4a16_dequant", "w4a16_gemm", "w4a16_gemm_ex",
-    "w4a16_gemm_host", "w4a16_gemm_static_ws", "w4a16_device_status",
+    "w4a16_gemm_host", "w4a16_gemm_static_ws", "w4a16_device_status", "w4a16_selftest_wait_timeout",
 )
 
 _lib = None
@@ -75,6 +75,8 @@ def load():
     L.w4a16_gemm_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.w4a16_gemm_static_ws.restype = i
     L.w4a16_gemm_static_ws.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    L.w4a16_selftest_wait_timeout.restype = i
+    L.w4a16_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
     L.w4a16_device_status.restype = i
     L.w4a16_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
     _lib = L
@@ -138,6 +140,11 @@ def w4a16_device_status() -> int:
     if rc not in (0, -8):
         raise W4A16Error(rc, "w4a16_device_status")
     return v.value
+
+
+def w4a16_selftest_wait_timeout(limit_us: int = 1000) -> None:
+    """Enqueue the diagnostic kernel whose bounded wait runs out (see ``w4a16_device_status``)."""
+    _check(load().w4a16_selftest_wait_timeout(int(limit_us), _stream()), "w4a16_selftest_wait_timeout")
 
 
 # ------------------------------------------------------------------ operations

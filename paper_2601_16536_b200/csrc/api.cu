@@ -5,6 +5,8 @@
 
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "kernels_basic.cuh"
 #include "kernel_decode.cuh"
@@ -28,13 +30,40 @@ struct DeviceState {
     bool decode_attr_set[3][4][2] = {};   // [mb][CTAs per SM][cluster exchange]
     bool tile_attr_set[5] = {false, false, false, false, false};
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
-    // kernel in its stream has finished.  After w4a16_pack was enqueued the next GEMM launch is
-    // therefore a plain, fully ordered one (it runs after the pack kernels), and only the launches
-    // after it overlap their predecessor again.
-    bool pdl_ok = false;
+    // kernel in its stream has finished.  The previous kernel of a stream may be a w4a16_pack that
+    // writes those weights, so the first GEMM launched on a stream after any pack on the device is a
+    // plain, fully ordered launch, and only the launches after it on that stream overlap their
+    // predecessor again.  pack_epoch counts the packs; the table remembers, per stream, the epoch of
+    // its last GEMM launch (a stream that is not in the table gets a plain launch).
+    unsigned long long pack_epoch = 1;
+    struct StreamEpoch { cudaStream_t stream; unsigned long long epoch; };
+    static constexpr int kStreamSlots = 32;
+    StreamEpoch streams[kStreamSlots] = {};
+    int stream_evict = 0;
     bool cluster_ok = true;   // cleared when a cluster launch is refused (fewer SMs than usual, MPS limits ...)
+
+    // May this launch on `st` overlap the previous kernel of the stream?  Records the launch.
+    bool pdl_allowed(cudaStream_t st) {
+        for (int i = 0; i < kStreamSlots; ++i) {
+            if (streams[i].epoch != 0 && streams[i].stream == st) {
+                const bool ok = streams[i].epoch == pack_epoch;
+                streams[i].epoch = pack_epoch;
+                return ok;
+            }
+        }
+        int slot = -1;
+        for (int i = 0; i < kStreamSlots; ++i)
+            if (streams[i].epoch == 0) { slot = i; break; }
+        if (slot < 0) { slot = stream_evict; stream_evict = (stream_evict + 1) % kStreamSlots; }
+        streams[slot].stream = st;
+        streams[slot].epoch = pack_epoch;
+        return false;
+    }
 };
 DeviceState g_dev[kMaxDevices];
+// One lock for the per-device records above (workspace registration, attribute flags, stream table):
+// the entry points may be called from several host threads.
+std::mutex g_mu;
 
 int current_device(DeviceState** out) {
     int dev = -1;
@@ -388,6 +417,7 @@ size_t w4a16_packed_z_bytes(int N, int K, int group) {
 }
 
 int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return 1;
     int G = K / group;
     switch (resolve_path(M, N, G, 0, sm_count_or_default(), path, cluster_ok_or_default())) {
@@ -397,6 +427,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
     }
 }
 int w4a16_choose_path(int M, int N, int K, int group) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return W4A16_ERR_SHAPE;
     return resolve_path(M, N, K / group, 0, sm_count_or_default(), W4A16_PATH_AUTO, cluster_ok_or_default());
 }
@@ -405,12 +436,16 @@ int w4a16_choose_split_k(int M, int N, int K, int group) {
 }
 
 size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1 || split_k < 0 || split_k > K / group) return 0;
     // enough for whichever path w4a16_gemm / w4a16_gemm_ex may take with this split_k
     size_t need = 0;
     if (split_k != 1) {
-        DecodeGeom g = decode_geom(M, N, K / group, split_k, sm_count_or_default());
+        // the schedule differs between a device that places clusters and one that refused them: cover both
+        DecodeGeom g = decode_geom(M, N, K / group, split_k, sm_count_or_default(), true);
+        DecodeGeom g2 = decode_geom(M, N, K / group, split_k, sm_count_or_default(), false);
         need = decode_partial_bytes(g);
+        if (g2.split_k != 1 && decode_partial_bytes(g2) > need) need = decode_partial_bytes(g2);
         int s = split_k == 0 ? choose_split_decode(M, N, K / group, sm_count_or_default()) : split_k;
         size_t simple = simple_partial_bytes(M, N, s);
         if (simple > need) need = simple;
@@ -421,6 +456,7 @@ size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k) {
 }
 
 int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
+    std::lock_guard<std::mutex> lock(g_mu);
     DeviceState* d = nullptr;
     int rc = current_device(&d);
     if (rc != W4A16_OK) return rc;
@@ -443,6 +479,7 @@ int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
 
 int w4a16_pack(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_raw, void* Wq, void* S, void* Z,
                int N, int K, int group, w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (!Wq_raw || !S_raw || !Z_raw || !Wq || !S || !Z) return W4A16_ERR_NULL;
     int rc = check_weight_shape(N, K, group);
     if (rc != W4A16_OK) return rc;
@@ -458,12 +495,13 @@ int w4a16_pack(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_r
     pack_wq_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(Wq_raw, static_cast<uint32_t*>(Wq), N, G, words);
     pack_s_kernel<<<(unsigned)((sc + 255) / 256), 256, 0, st>>>(S_raw, static_cast<uint16_t*>(S), N, G, sc);
     pack_z_kernel<<<(unsigned)((zw + 255) / 256), 256, 0, st>>>(Z_raw, static_cast<uint32_t*>(Z), N, G, zw);
-    d->pdl_ok = false;
+    ++d->pack_epoch;
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
 int w4a16_dequant(const void* Wq, const void* S, const void* Z, uint16_t* W16, int N, int K, int group,
                   w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (!Wq || !S || !Z || !W16) return W4A16_ERR_NULL;
     int rc = check_weight_shape(N, K, group);
     if (rc != W4A16_OK) return rc;
@@ -478,8 +516,12 @@ int w4a16_dequant(const void* Wq, const void* S, const void* Z, uint16_t* W16, i
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
-int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
-                  int group, int split_k, int path, w4a16_stream_t stream) {
+}  // extern "C"
+
+namespace {
+// The body of w4a16_gemm_ex; the caller holds g_mu.
+int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
+                int group, int split_k, int path, w4a16_stream_t stream) {
     if (!A || !Wq || !S || !Z || !C) return W4A16_ERR_NULL;
     int rc = check_weight_shape(N, K, group);
     if (rc != W4A16_OK) return rc;
@@ -565,8 +607,7 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = d->pdl_ok ? 1 : 0;
-        d->pdl_ok = true;
+        cfg.numAttrs = d->pdl_allowed(st) ? 1 : 0;
         if (cudaLaunchKernelEx(&cfg, kern, tmap, p) != cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
@@ -593,10 +634,8 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
     p.nchunks = g.nchunks;
     p.stages = g.stages;
     void (*kern)(const DecodeParams) =
-        g.cluster ? ((g.mb == 2) ? gemm_decode_kernel<2, 2, true>
-                                 : (g.cps == 3) ? gemm_decode_kernel<1, 3, true> : gemm_decode_kernel<1, 2, true>)
-                  : ((g.mb == 2) ? gemm_decode_kernel<2, 2, false>
-                                 : (g.cps == 3) ? gemm_decode_kernel<1, 3, false> : gemm_decode_kernel<1, 2, false>);
+        g.cluster ? ((g.mb == 2) ? gemm_decode_kernel<2, 2, true> : gemm_decode_kernel<1, 2, true>)
+                  : ((g.mb == 2) ? gemm_decode_kernel<2, 2, false> : gemm_decode_kernel<1, 2, false>);
     if (!d->decode_attr_set[g.mb][g.cps][g.cluster ? 1 : 0]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
@@ -621,25 +660,33 @@ int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* 
         attr[n_attr].val.clusterDim.z = 1;
         ++n_attr;
     }
-    if (d->pdl_ok) {
+    if (d->pdl_allowed(st)) {
         attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
         ++n_attr;
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    d->pdl_ok = true;
     if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) {
         cudaGetLastError();
         if (g.cluster) {
             // the device would not place the clusters: from now on the workspace exchange (and the path
             // rule that goes with it), starting with this call
             d->cluster_ok = false;
-            return w4a16_gemm_ex(A, Wq, S, Z, C, M, N, K, group, split_k, path_asked, stream);
+            return gemm_locked(A, Wq, S, Z, C, M, N, K, group, split_k, path_asked, stream);
         }
         return W4A16_ERR_CUDA;
     }
     return W4A16_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
+                  int group, int split_k, int path, w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    return gemm_locked(A, Wq, S, Z, C, M, N, K, group, split_k, path, stream);
 }
 
 int w4a16_gemm(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
@@ -668,6 +715,7 @@ int w4a16_gemm_host(const uint16_t* A_host, uint16_t* A_dev, const void* Wq, con
 
 int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N,
                          int K, int group, int split_k, w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (!A || !Wq || !S || !Z || !C) return W4A16_ERR_NULL;
     int rc = check_weight_shape(N, K, group);
     if (rc != W4A16_OK) return rc;
@@ -684,8 +732,10 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     const DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, false);   // no clusters here: this entry point keeps the path it was built with
     if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
     if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
-    // the whole scratch need of this shape must fit the built-in array, or nothing is launched
-    if (kWsHeaderBytes + decode_partial_bytes(g) > (size_t)W4A16_STATIC_WS_BYTES) return W4A16_ERR_WORKSPACE;
+    // the whole scratch need of this shape must fit the built-in array, or nothing is launched (a schedule of
+    // whole tiles, split_k == 1, leaves no partial tiles and draws no tickets: it needs none)
+    if (g.split_k != 1 && kWsHeaderBytes + decode_partial_bytes(g) > (size_t)W4A16_STATIC_WS_BYTES)
+        return W4A16_ERR_WORKSPACE;
 
     // first call on this device: resolve the array's device address (this device is current)
     if (g_static_ws_addr[dev] == nullptr) {
@@ -715,8 +765,7 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2, false>
-                            : (g.cps == 3) ? gemm_decode_kernel<1, 3, false> : gemm_decode_kernel<1, 2, false>;
+    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2, false> : gemm_decode_kernel<1, 2, false>;
     if (!d->decode_attr_set[g.mb][g.cps][0]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
@@ -729,7 +778,20 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
+int w4a16_selftest_wait_timeout(unsigned limit_us, w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (limit_us < 1 || limit_us > 100000) return W4A16_ERR_SHAPE;
+    DeviceState* d = nullptr;
+    int rc = current_device(&d);
+    if (rc != W4A16_OK) return rc;
+    if (!d->is_sm100) return W4A16_ERR_ARCH;
+    wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>((unsigned long long)limit_us * 1000ull,
+                                                                               nullptr);
+    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
+}
+
 int w4a16_device_status(int* status_out) {
+    std::lock_guard<std::mutex> lock(g_mu);
     if (!status_out) return W4A16_ERR_NULL;
     int v = 0, zero = 0;
     if (cudaDeviceSynchronize() != cudaSuccess ||
@@ -739,6 +801,16 @@ int w4a16_device_status(int* status_out) {
         return W4A16_ERR_CUDA;
     }
     *status_out = v;
+    if (v != 0) {
+        // a kernel that gave up returned before it drew its tickets: the counters of the registered
+        // workspace may be non-zero, and the next call would take a tile for complete too early
+        DeviceState* d = nullptr;
+        if (current_device(&d) == W4A16_OK && d->ws != nullptr &&
+            (cudaMemset(d->ws, 0, kWsFullHeaderBytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)) {
+            cudaGetLastError();
+            return W4A16_ERR_CUDA;
+        }
+    }
     return v == 0 ? W4A16_OK : W4A16_ERR_DEVICE_STATUS;
 }
 

@@ -47,8 +47,7 @@ __host__ __device__ constexpr int block_word_index(int col, int kw) {
 // Status word: a kernel whose bounded wait runs out ORs a code in here and returns.
 __device__ int g_status_word = 0;
 constexpr int kStatusMbarTimeout = 1;
-constexpr int kStatusTmemAlloc = 2;
-constexpr int kStatusTicket = 4;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every bounded wait of the GEMM kernels: two seconds
 
 __device__ __forceinline__ void report_status(int code) { atomicOr(&g_status_word, code); }
 
@@ -78,7 +77,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // complete).  Slow path: try_wait with a suspend-time hint, so that a waiting warp sleeps in the
 // barrier unit instead of spending issue slots on polling, and a wall-clock limit read from
 // %globaltimer (the hint is only a hint: an iteration count would not bound the time).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs) {
     uint32_t ok;
     asm volatile(
         "{\n\t"
@@ -105,7 +104,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if (ok) return true;
         unsigned long long t1;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-        if (t1 - t0 > 2000000000ull) break;
+        if (t1 - t0 > limit_ns) break;
     }
     report_status(kStatusMbarTimeout);
     return false;
@@ -130,7 +129,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
         if (ok) return true;
         unsigned long long t1;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-        if (t1 - t0 > 2000000000ull) break;
+        if (t1 - t0 > kWaitLimitNs) break;
     }
     report_status(kStatusMbarTimeout);
     return false;

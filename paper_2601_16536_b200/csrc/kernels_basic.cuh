@@ -153,4 +153,18 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ ws, __half* __res
     C[i] = __float2half_rn(acc);
 }
 
+// Diagnostic: one warp waits on a barrier that nobody ever arrives on, with a limit of `limit_ns`.  The wait
+// runs out, records kStatusMbarTimeout in the status word and the kernel returns normally: the same exit
+// every GEMM kernel takes when one of its waits gives up, exercised without any fault.
+__global__ void wait_timeout_probe_kernel(unsigned long long limit_ns, int* gave_up) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(&bar, 0u, limit_ns);
+    if (threadIdx.x == 0 && gave_up != nullptr) *gave_up = ok ? 0 : 1;
+}
+
 }  // namespace w4a16

@@ -29,7 +29,7 @@ def c_f64(C: torch.Tensor) -> np.ndarray:
 
 
 def assert_close(C_gpu: np.ndarray, C_ref: np.ndarray, what=""):
-    """spec tolerances against the FP64 oracle."""
+    """Relative Frobenius error <= REL_FROB_TOL and every element within ELEM_TOL (1 + |C_ref|) of the FP64 oracle."""
     mask = ~np.isnan(C_ref)
     g, r = C_gpu[mask], C_ref[mask]
     assert np.all(np.isfinite(g)), what

@@ -8,10 +8,10 @@ import sys
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _run(env_extra=None):
+def _run(env_extra=None, gpus=1):
     env = dict(os.environ)
     env.update(env_extra or {})
-    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", str(gpus),
                           "--steps", "1", "--warmup", "0"], capture_output=True, text=True, env=env, timeout=600)
     assert out.returncode == 0, out.stderr
     return out.stdout.strip()
@@ -31,4 +31,11 @@ def test_reference_arm_prints_the_contract_line():
 
 
 def test_reference_arm_is_silent_on_other_ranks():
-    assert _run({"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1"}) == ""
+    assert _run({"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1"}, gpus=2) == ""
+
+
+def test_gpus_must_match_the_launched_world_size():
+    env = dict(os.environ, RANK="0", WORLD_SIZE="2", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "4",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, env=env, timeout=600)
+    assert out.returncode != 0 and "WORLD_SIZE" in out.stderr

@@ -1,7 +1,7 @@
 """GPU parity of w4a16_gemm against the FP64 oracle (Eq. 2; Algorithm 1 Split-K), through the C ABI.
 
-Tolerances (stated by the benchmark spec): relative Frobenius error <= 1e-3 and per element
-|dC| <= 2e-3 (1 + |C_ref|).  With exactly representable inputs the result is unique and must be
+Tolerances: relative Frobenius error <= 1e-3 and per element |dC| <= 2e-3 (1 + |C_ref|) against the
+FP64-accumulated oracle.  With exactly representable inputs the result is unique and must be
 bit-equal for every path and split.
 """
 import numpy as np

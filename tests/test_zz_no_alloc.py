@@ -37,8 +37,14 @@ def test_static_scratch_matches_the_workspace_entry_point_twice(M, K, N, split_k
     results = []
     for call in range(2):
         C.fill_(float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         B.w4a16_gemm_static_ws(A, pw, C, split_k=split_k)
         torch.cuda.synchronize()
+        if call == 1:
+            # the entry point's one promise: no device memory is taken.  (The first call of a process may
+            # load the kernel's code; the second finds everything in place.)
+            assert torch.cuda.mem_get_info()[0] == free_before
         assert B.w4a16_device_status() == 0
         # same tolerances as the other GEMM parity tests, against the existing entry point ...
         assert_close(c_f64(C), c_f64(want), "static scratch vs workspace, call %d" % call)
@@ -46,6 +52,21 @@ def test_static_scratch_matches_the_workspace_entry_point_twice(M, K, N, split_k
         assert_close(c_f64(C), ref, "static scratch vs oracle, call %d" % call)
         results.append(c_bits(C).copy())
     assert np.array_equal(results[0], results[1])
+
+
+def test_whole_tile_schedules_need_no_scratch_however_wide():
+    # N = 128256 (2004 column tiles): the library deals whole tiles, which leave no partial tiles and draw no
+    # tickets, so the shape runs although 2004 partial-tile slots would not fit the built-in array
+    M, K, N = 1, 1024, 128256
+    d = wl.make_problem(M, K, N, seed=11)
+    pw = pack_problem(d, N, K)
+    A = to_dev(d["A"])
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+    for split_k in (0, 1):
+        C = B.w4a16_gemm_static_ws(A, pw, split_k=split_k)
+        torch.cuda.synchronize()
+        assert B.w4a16_device_status() == 0
+        assert_close(c_f64(C), ref, "wide N, split_k %d" % split_k)
 
 
 def test_static_scratch_rejects_what_does_not_fit():
