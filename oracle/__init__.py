@@ -145,5 +145,20 @@ def gemm_int(A_int, Wq, E, Z, M, N, K, group=128) -> np.ndarray:
     return C
 
 
+def epilogue(C_ref: np.ndarray, bias=None, act: str = "none") -> np.ndarray:
+    """The optional step after the product (outside the paper's Algorithm 1), in FP64:
+    y = act(C_ref + bias[n]) with act in {"none", "relu": max(x, 0), "silu": x / (1 + exp(-x))}."""
+    y = np.array(C_ref, dtype=np.float64, copy=True)
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)[None, :]
+    if act == "relu":
+        y = np.maximum(y, 0.0)
+    elif act == "silu":
+        y = y / (1.0 + np.exp(-y))
+    elif act != "none":
+        raise ValueError(act)
+    return y
+
+
 def num_threads() -> int:
     return int(lib().orc_num_threads())
