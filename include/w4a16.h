@@ -4,9 +4,12 @@
  *     C[M,N] = A[M,K] . Dequant(W)[K,N],   Dequant(W) = s (W - z)        (paper Eq. 2)
  *
  * A is FP16, W is unsigned INT4 (0..15) with one FP16 scale s and one integer zero
- * point z (0..15) per group of `group` = 128 consecutive k and per column n,
+ * point z (0..15) per group of `group` consecutive k (128, 64 or 32) and per column n,
  * accumulation is FP32 and C is FP16 (Algorithm 1: dequantize, Split-K multiply,
- * reduce + FP32->FP16 cast).
+ * reduce + FP32->FP16 cast).  The *_fmt entry points add the format variants the paper
+ * names without fixing them: symmetric quantization (Eq. 1 with the zero point fixed, here
+ * z = 8 for the unsigned nibbles, i.e. q - 8 in -8 .. 7, and no Z buffer) and BF16 instead of
+ * FP16 for activations, scales, dequantized weights and output (Section 1).
  *
  * General rules
  *   - Every pointer is a DEVICE pointer owned by the caller unless a parameter says
@@ -28,9 +31,9 @@
  *   Z_raw   uint8  [K/group, N] row-major, one zero point (0..15) per byte
  * Packed layout (what the kernels consume): opaque; sizes from w4a16_packed_*_bytes.
  *
- * Preconditions shared by pack / dequant / gemm:  group == 128, K > 0, K % 128 == 0,
- * N > 0, N % 64 == 0; all buffers 16-byte aligned.  Violations -> W4A16_ERR_SHAPE /
- * W4A16_ERR_ALIGN / W4A16_ERR_NULL.
+ * Preconditions shared by pack / dequant / gemm:  group in {32, 64, 128}, K > 0,
+ * K % 128 == 0, N > 0, N % 64 == 0; all buffers 16-byte aligned.  Violations ->
+ * W4A16_ERR_SHAPE / W4A16_ERR_ALIGN / W4A16_ERR_NULL.
  */
 #ifndef W4A16_H_
 #define W4A16_H_
@@ -49,7 +52,7 @@ enum {
     W4A16_ERR_NULL = -1,          /* a required pointer is NULL */
     W4A16_ERR_SHAPE = -2,         /* M, N, K or group outside the supported set */
     W4A16_ERR_ALIGN = -3,         /* a buffer is not 16-byte aligned */
-    W4A16_ERR_SPLITK = -4,        /* split_k < 0 or > K/group */
+    W4A16_ERR_SPLITK = -4,        /* split_k < 0 or > K/128 */
     W4A16_ERR_WORKSPACE = -5,     /* split_k > 1 needs more workspace than was set */
     W4A16_ERR_CUDA = -6,          /* a CUDA runtime call failed (launch, attribute, copy) */
     W4A16_ERR_ARCH = -7,          /* current device is not sm_100 */
@@ -64,6 +67,19 @@ enum {
     W4A16_PATH_DECODE = 2, /* small-M bandwidth-bound kernel (M <= 64): TMA bulk staging,
                               in-register unpack, warp-level tensor-core MMA */
     W4A16_PATH_TILE = 3    /* tcgen05 / TMEM tile kernel, any M (batch tiles of 16 .. 256 rows) */
+};
+
+/* Format options of the *_fmt entry points (bit flags). */
+enum {
+    W4A16_FLAG_SYMMETRIC = 1, /* zero point 8 for every weight; Z pointers are ignored and may be NULL */
+    W4A16_FLAG_BF16 = 2       /* A, S, the dequantized weights and C are BF16 instead of FP16 */
+};
+
+/* Optional step fused into the final cast of w4a16_gemm_fmt (not part of Algorithm 1). */
+enum {
+    W4A16_ACT_NONE = 0,
+    W4A16_ACT_RELU = 1, /* max(x, 0) */
+    W4A16_ACT_SILU = 2  /* x / (1 + exp(-x)) */
 };
 
 const char *w4a16_strerror(int code);
@@ -116,8 +132,9 @@ int w4a16_dequant(const void *Wq, const void *S, const void *Z, uint16_t *W16,
  *   A   FP16 [M, K] row-major (K contiguous), M >= 1
  *   Wq, S, Z   packed buffers from w4a16_pack
  *   C   FP16 [M, N] row-major, fully overwritten (no beta)
- *   split_k   0 = automatic, else 1 <= split_k <= K/group (some paths cap it lower and
- *             return W4A16_ERR_SPLITK beyond their cap)
+ *   split_k   0 = automatic, else 1 <= split_k <= K/128: slices are whole blocks of 128 k,
+ *             i.e. whole groups for every supported group size (some paths cap it lower
+ *             and return W4A16_ERR_SPLITK beyond their cap)
  * Results are bit-identical from run to run for fixed arguments (with split_k == 0 the schedule,
  * and with it the order of the FP32 sums, is the library's choice for this entry point and device;
  * it changes once, for good, if the device refuses a thread-block-cluster launch).  If the chosen
@@ -135,6 +152,26 @@ int w4a16_gemm(const uint16_t *A, const void *Wq, const void *S, const void *Z, 
  * W4A16_ERR_PATH if that path does not support the shape. */
 int w4a16_gemm_ex(const uint16_t *A, const void *Wq, const void *S, const void *Z, uint16_t *C,
                   int M, int N, int K, int group, int split_k, int path, w4a16_stream_t stream);
+
+/* The same three operations with the format options above (flags = 0 and act = W4A16_ACT_NONE,
+ * bias = NULL give exactly w4a16_pack / w4a16_dequant / w4a16_gemm_ex).
+ *   W4A16_FLAG_SYMMETRIC   Eq. 1's symmetric case: every zero point is 8; Z_raw / Z are not read
+ *                          and no Z traffic exists (pass NULL).
+ *   W4A16_FLAG_BF16        S_raw / S, A, W16 and C hold BF16 bit patterns; the dequantized weight
+ *                          is bf16_rn((q - z) * s), accumulation stays FP32, one FP32->BF16
+ *                          rounding at the end.  (pack only moves 16-bit scales: the flag does
+ *                          not change it.)
+ *   bias   NULL, or [N] values in C's 16-bit format added to the FP32 sum before `act` and the
+ *          final rounding:  C[m, n] = rn16(act(sum + bias[n])).
+ * Everything else (layouts, split_k, path, ordering, error codes) is as documented above. */
+int w4a16_pack_fmt(const uint32_t *Wq_raw, const uint16_t *S_raw, const uint8_t *Z_raw,
+                   void *Wq, void *S, void *Z, int N, int K, int group, int flags,
+                   w4a16_stream_t stream);
+int w4a16_dequant_fmt(const void *Wq, const void *S, const void *Z, uint16_t *W16,
+                      int N, int K, int group, int flags, w4a16_stream_t stream);
+int w4a16_gemm_fmt(const uint16_t *A, const void *Wq, const void *S, const void *Z,
+                   const uint16_t *bias, uint16_t *C, int M, int N, int K, int group,
+                   int split_k, int path, int flags, int act, w4a16_stream_t stream);
 
 /* End-to-end form of w4a16_gemm for callers whose activations live in HOST memory:
  * copies A_host (FP16 [M, K], ideally pinned) into the caller's device staging buffer

@@ -18,6 +18,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libw4a16.so")
 
 PATH_AUTO, PATH_SIMPLE, PATH_DECODE, PATH_TILE = 0, 1, 2, 3
+FLAG_SYMMETRIC, FLAG_BF16 = 1, 2
+ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
 GROUP = 128
 WS_HEADER_BYTES = 16384 + 131072   # W4A16_WORKSPACE_HEADER_BYTES
 
@@ -26,6 +28,7 @@ EXPORTS = (
     "w4a16_workspace_bytes", "w4a16_set_workspace", "w4a16_choose_split_k",
     "w4a16_choose_split_k_ex", "w4a16_choose_path", "w4a16_pack", "w4a16_dequant", "w4a16_gemm", "w4a16_gemm_ex",
     "w4a16_gemm_host", "w4a16_gemm_static_ws", "w4a16_device_status", "w4a16_selftest_wait_timeout",
+    "w4a16_pack_fmt", "w4a16_dequant_fmt", "w4a16_gemm_fmt",
 )
 
 _lib = None
@@ -75,6 +78,12 @@ def load():
     L.w4a16_gemm_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.w4a16_gemm_static_ws.restype = i
     L.w4a16_gemm_static_ws.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    L.w4a16_pack_fmt.restype = i
+    L.w4a16_pack_fmt.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp]
+    L.w4a16_dequant_fmt.restype = i
+    L.w4a16_dequant_fmt.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
+    L.w4a16_gemm_fmt.restype = i
+    L.w4a16_gemm_fmt.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp]
     L.w4a16_selftest_wait_timeout.restype = i
     L.w4a16_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
     L.w4a16_device_status.restype = i
@@ -150,44 +159,67 @@ def w4a16_selftest_wait_timeout(limit_us: int = 1000) -> None:
 # ------------------------------------------------------------------ operations
 @dataclass
 class PackedWeights:
-    Wq: torch.Tensor   # uint8, opaque
-    S: torch.Tensor    # uint8, opaque
-    Z: torch.Tensor    # uint8, opaque
+    Wq: torch.Tensor             # uint8, opaque
+    S: torch.Tensor              # uint8, opaque
+    Z: Optional[torch.Tensor]    # uint8, opaque; None for a symmetric format
     N: int
     K: int
     group: int = GROUP
+    flags: int = 0               # FLAG_SYMMETRIC | FLAG_BF16
 
 
-def w4a16_pack(Wq_raw: torch.Tensor, S_raw: torch.Tensor, Z_raw: torch.Tensor,
-               N: int, K: int, group: int = GROUP) -> PackedWeights:
-    """Raw int32/uint32 [K/8,N], fp16 [K/group,N], uint8 [K/group,N] CUDA tensors -> packed."""
+def _dtype_of(flags: int):
+    return torch.bfloat16 if flags & FLAG_BF16 else torch.float16
+
+
+def w4a16_pack(Wq_raw: torch.Tensor, S_raw: torch.Tensor, Z_raw: Optional[torch.Tensor],
+               N: int, K: int, group: int = GROUP, flags: int = 0) -> PackedWeights:
+    """Raw int32/uint32 [K/8,N], 16-bit scales [K/group,N], uint8 [K/group,N] (None when symmetric)
+    CUDA tensors -> packed.  ``flags == 0`` goes through ``w4a16_pack``, anything else through
+    ``w4a16_pack_fmt``."""
     dev = Wq_raw.device
+    sym = bool(flags & FLAG_SYMMETRIC)
     nb = (w4a16_packed_wq_bytes(N, K, group), w4a16_packed_s_bytes(N, K, group),
-          w4a16_packed_z_bytes(N, K, group))
+          0 if sym else w4a16_packed_z_bytes(N, K, group))
     if nb[0] == 0:
         raise W4A16Error(-2, "w4a16_pack")
-    out = [torch.empty(b, dtype=torch.uint8, device=dev) for b in nb]
-    _check(load().w4a16_pack(_ptr(Wq_raw), _ptr(S_raw), _ptr(Z_raw), _ptr(out[0]), _ptr(out[1]),
-                             _ptr(out[2]), N, K, group, _stream()), "w4a16_pack")
-    return PackedWeights(out[0], out[1], out[2], N, K, group)
+    out = [torch.empty(b, dtype=torch.uint8, device=dev) if b else None for b in nb]
+    if flags == 0:
+        _check(load().w4a16_pack(_ptr(Wq_raw), _ptr(S_raw), _ptr(Z_raw), _ptr(out[0]), _ptr(out[1]),
+                                 _ptr(out[2]), N, K, group, _stream()), "w4a16_pack")
+    else:
+        _check(load().w4a16_pack_fmt(_ptr(Wq_raw), _ptr(S_raw), None if sym else _ptr(Z_raw), _ptr(out[0]),
+                                     _ptr(out[1]), _ptr(out[2]), N, K, group, flags, _stream()), "w4a16_pack_fmt")
+    return PackedWeights(out[0], out[1], out[2], N, K, group, flags)
 
 
 def w4a16_dequant(pw: PackedWeights, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     if out is None:
-        out = torch.empty((pw.K, pw.N), dtype=torch.float16, device=pw.Wq.device)
-    _check(load().w4a16_dequant(_ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(out), pw.N, pw.K, pw.group,
-                                _stream()), "w4a16_dequant")
+        out = torch.empty((pw.K, pw.N), dtype=_dtype_of(pw.flags), device=pw.Wq.device)
+    if pw.flags == 0:
+        _check(load().w4a16_dequant(_ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(out), pw.N, pw.K, pw.group,
+                                    _stream()), "w4a16_dequant")
+    else:
+        _check(load().w4a16_dequant_fmt(_ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(out), pw.N, pw.K, pw.group,
+                                        pw.flags, _stream()), "w4a16_dequant_fmt")
     return out
 
 
 def w4a16_gemm(A: torch.Tensor, pw: PackedWeights, C: Optional[torch.Tensor] = None,
-               split_k: int = 0, path: int = PATH_AUTO) -> torch.Tensor:
-    """C[M,N] = A[M,K] . Dequant(W); A fp16 CUDA tensor, row-major contiguous."""
+               split_k: int = 0, path: int = PATH_AUTO, bias: Optional[torch.Tensor] = None,
+               act: int = ACT_NONE) -> torch.Tensor:
+    """C[M,N] = A[M,K] . Dequant(W); A a 16-bit CUDA tensor (FP16, or BF16 for a BF16 format), row-major
+    contiguous.  Plain formats go through ``w4a16_gemm_ex``; format flags, ``bias`` or ``act`` through
+    ``w4a16_gemm_fmt``."""
     M = A.shape[0]
     if C is None:
-        C = torch.empty((M, pw.N), dtype=torch.float16, device=A.device)
-    _check(load().w4a16_gemm_ex(_ptr(A), _ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(C), M, pw.N, pw.K,
-                                pw.group, split_k, path, _stream()), "w4a16_gemm")
+        C = torch.empty((M, pw.N), dtype=_dtype_of(pw.flags), device=A.device)
+    if pw.flags == 0 and bias is None and act == ACT_NONE:
+        _check(load().w4a16_gemm_ex(_ptr(A), _ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(C), M, pw.N, pw.K,
+                                    pw.group, split_k, path, _stream()), "w4a16_gemm")
+    else:
+        _check(load().w4a16_gemm_fmt(_ptr(A), _ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z), _ptr(bias), _ptr(C), M, pw.N,
+                                     pw.K, pw.group, split_k, path, pw.flags, act, _stream()), "w4a16_gemm_fmt")
     return C
 
 

@@ -27,8 +27,8 @@ struct DeviceState {
     int max_smem_optin = 0;
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    bool decode_attr_set[3][4][2] = {};   // [mb][CTAs per SM][cluster exchange]
-    bool tile_attr_set[5] = {false, false, false, false, false};
+    bool decode_attr_set[3][2][3][2] = {};   // [mb][cluster exchange][log2 SG][bf16]
+    bool tile_attr_set[5][3][2] = {};         // [batch-tile index][log2 SG][bf16]
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
     // kernel in its stream has finished.  The previous kernel of a stream may be a w4a16_pack that
     // writes those weights, so the first GEMM launched on a stream after any pack on the device is a
@@ -92,10 +92,12 @@ int current_device(DeviceState** out) {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_weight_shape(int N, int K, int group) {
-    if (group != kGroup) return W4A16_ERR_SHAPE;
+    if (!group_ok(group)) return W4A16_ERR_SHAPE;
     if (K <= 0 || N <= 0 || K % kGroup != 0 || N % kTileN != 0) return W4A16_ERR_SHAPE;
     return W4A16_OK;
 }
+int log2_sg(int sg) { return sg == 1 ? 0 : sg == 2 ? 1 : 2; }
+bool flags_ok(int flags) { return (flags & ~(W4A16_FLAG_SYMMETRIC | W4A16_FLAG_BF16)) == 0; }
 
 size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 
@@ -124,7 +126,7 @@ struct DecodeGeom {
     int split_k;   // what the kernel runs: 0 = balanced chunks, S >= 1 = S slices per tile
 };
 
-DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_cluster = true) {
+DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_cluster = true, int sg = 1) {
     DecodeGeom g;
     g.mb = decode_mb(M);
     g.mchunks = (M + 8 * g.mb - 1) / (8 * g.mb);
@@ -186,11 +188,11 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     g.cluster = allow_cluster && split_k >= 2 && split_k <= kDecMaxCluster && g.nchunks == g.ctas && g.mchunks == 1;
     const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
     const int xs = g.cluster ? split_k : 0;   // slices that meet in the exchange buffer
-    int st = (budget - 128 - decode_red_bytes(g.mb) - decode_xch_bytes(g.mb, xs)) / decode_stage_bytes(g.mb);
+    int st = (budget - 128 - decode_red_bytes(g.mb) - decode_xch_bytes(g.mb, xs)) / decode_stage_bytes(g.mb, sg);
     if (st > kDecMaxStages) st = kDecMaxStages;
     if (st < 2) st = 2;
     g.stages = st;
-    g.smem_bytes = decode_smem_bytes(g.mb, st, xs);
+    g.smem_bytes = decode_smem_bytes(g.mb, sg, st, xs);
     return g;
 }
 
@@ -391,7 +393,7 @@ const char* w4a16_strerror(int code) {
     switch (code) {
         case W4A16_OK: return "ok";
         case W4A16_ERR_NULL: return "null pointer argument";
-        case W4A16_ERR_SHAPE: return "unsupported shape (need group == 128, K % 128 == 0, N % 64 == 0, M >= 1)";
+        case W4A16_ERR_SHAPE: return "unsupported shape or option (need group in {32, 64, 128}, K % 128 == 0, N % 64 == 0, M >= 1)";
         case W4A16_ERR_ALIGN: return "buffer not 16-byte aligned (workspace: 256-byte)";
         case W4A16_ERR_SPLITK: return "split_k out of range for this shape / path";
         case W4A16_ERR_WORKSPACE: return "split-K workspace missing or too small (w4a16_set_workspace)";
@@ -411,7 +413,7 @@ size_t w4a16_packed_s_bytes(int N, int K, int group) {
     if (check_weight_shape(N, K, group) != W4A16_OK) return 0;
     return (size_t)(K / group) * (size_t)N * 2;
 }
-size_t w4a16_packed_z_bytes(int N, int K, int group) {
+size_t w4a16_packed_z_bytes(int N, int K, int group) {   // asymmetric formats; a symmetric one has no Z buffer
     if (check_weight_shape(N, K, group) != W4A16_OK) return 0;
     return (size_t)(K / group) * (size_t)N / 2;
 }
@@ -419,7 +421,7 @@ size_t w4a16_packed_z_bytes(int N, int K, int group) {
 int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return 1;
-    int G = K / group;
+    int G = K / kGroup;
     switch (resolve_path(M, N, G, 0, sm_count_or_default(), path, cluster_ok_or_default())) {
         case W4A16_PATH_DECODE: return choose_split_decode(M, N, G, sm_count_or_default());
         case W4A16_PATH_TILE: return choose_split_tile(M, N, G, sm_count_or_default());
@@ -429,7 +431,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
 int w4a16_choose_path(int M, int N, int K, int group) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return W4A16_ERR_SHAPE;
-    return resolve_path(M, N, K / group, 0, sm_count_or_default(), W4A16_PATH_AUTO, cluster_ok_or_default());
+    return resolve_path(M, N, K / kGroup, 0, sm_count_or_default(), W4A16_PATH_AUTO, cluster_ok_or_default());
 }
 int w4a16_choose_split_k(int M, int N, int K, int group) {
     return w4a16_choose_split_k_ex(M, N, K, group, W4A16_PATH_AUTO);
@@ -437,19 +439,19 @@ int w4a16_choose_split_k(int M, int N, int K, int group) {
 
 size_t w4a16_workspace_bytes(int M, int N, int K, int group, int split_k) {
     std::lock_guard<std::mutex> lock(g_mu);
-    if (check_weight_shape(N, K, group) != W4A16_OK || M < 1 || split_k < 0 || split_k > K / group) return 0;
+    if (check_weight_shape(N, K, group) != W4A16_OK || M < 1 || split_k < 0 || split_k > K / kGroup) return 0;
     // enough for whichever path w4a16_gemm / w4a16_gemm_ex may take with this split_k
     size_t need = 0;
     if (split_k != 1) {
         // the schedule differs between a device that places clusters and one that refused them: cover both
-        DecodeGeom g = decode_geom(M, N, K / group, split_k, sm_count_or_default(), true);
-        DecodeGeom g2 = decode_geom(M, N, K / group, split_k, sm_count_or_default(), false);
+        DecodeGeom g = decode_geom(M, N, K / kGroup, split_k, sm_count_or_default(), true);
+        DecodeGeom g2 = decode_geom(M, N, K / kGroup, split_k, sm_count_or_default(), false);
         need = decode_partial_bytes(g);
         if (g2.split_k != 1 && decode_partial_bytes(g2) > need) need = decode_partial_bytes(g2);
-        int s = split_k == 0 ? choose_split_decode(M, N, K / group, sm_count_or_default()) : split_k;
+        int s = split_k == 0 ? choose_split_decode(M, N, K / kGroup, sm_count_or_default()) : split_k;
         size_t simple = simple_partial_bytes(M, N, s);
         if (simple > need) need = simple;
-        TileGeom tg = tile_geom(M, N, K / group, split_k, sm_count_or_default(), 227 * 1024);
+        TileGeom tg = tile_geom(M, N, K / kGroup, split_k, sm_count_or_default(), 227 * 1024);
         if (tile_workspace_bytes(tg) > need) need = tile_workspace_bytes(tg);
     }
     return need == 0 ? 0 : kWsFullHeaderBytes + need;
@@ -477,57 +479,112 @@ int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
     return W4A16_OK;
 }
 
-int w4a16_pack(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_raw, void* Wq, void* S, void* Z,
-               int N, int K, int group, w4a16_stream_t stream) {
+int w4a16_pack_fmt(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_raw, void* Wq, void* S, void* Z,
+                   int N, int K, int group, int flags, w4a16_stream_t stream) {
     std::lock_guard<std::mutex> lock(g_mu);
-    if (!Wq_raw || !S_raw || !Z_raw || !Wq || !S || !Z) return W4A16_ERR_NULL;
+    if (!flags_ok(flags)) return W4A16_ERR_SHAPE;
+    const bool sym = (flags & W4A16_FLAG_SYMMETRIC) != 0;
+    if (!Wq_raw || !S_raw || !Wq || !S) return W4A16_ERR_NULL;
+    if (!sym && (!Z_raw || !Z)) return W4A16_ERR_NULL;
     int rc = check_weight_shape(N, K, group);
     if (rc != W4A16_OK) return rc;
-    if (!aligned16(Wq_raw) || !aligned16(S_raw) || !aligned16(Z_raw) || !aligned16(Wq) || !aligned16(S) ||
-        !aligned16(Z))
-        return W4A16_ERR_ALIGN;
+    if (!aligned16(Wq_raw) || !aligned16(S_raw) || !aligned16(Wq) || !aligned16(S)) return W4A16_ERR_ALIGN;
+    if (!sym && (!aligned16(Z_raw) || !aligned16(Z))) return W4A16_ERR_ALIGN;
     DeviceState* d = nullptr;
     if ((rc = current_device(&d)) != W4A16_OK) return rc;
     if (!d->is_sm100) return W4A16_ERR_ARCH;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int G = K / group;
-    size_t words = (size_t)K * N / 8, sc = (size_t)G * N, zw = (size_t)G * N / 8;
+    const int G = K / kGroup, sg = kGroup / group;
+    size_t words = (size_t)K * N / 8, sc = (size_t)G * sg * N, zw = sc / 8;
     pack_wq_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(Wq_raw, static_cast<uint32_t*>(Wq), N, G, words);
-    pack_s_kernel<<<(unsigned)((sc + 255) / 256), 256, 0, st>>>(S_raw, static_cast<uint16_t*>(S), N, G, sc);
-    pack_z_kernel<<<(unsigned)((zw + 255) / 256), 256, 0, st>>>(Z_raw, static_cast<uint32_t*>(Z), N, G, zw);
+    pack_s_kernel<<<(unsigned)((sc + 255) / 256), 256, 0, st>>>(S_raw, static_cast<uint16_t*>(S), N, G, sg, sc);
+    if (!sym)
+        pack_z_kernel<<<(unsigned)((zw + 255) / 256), 256, 0, st>>>(Z_raw, static_cast<uint32_t*>(Z), N, G, sg, zw);
     ++d->pack_epoch;
+    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
+}
+
+int w4a16_pack(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_raw, void* Wq, void* S, void* Z,
+               int N, int K, int group, w4a16_stream_t stream) {
+    if (!Z_raw || !Z) return W4A16_ERR_NULL;
+    return w4a16_pack_fmt(Wq_raw, S_raw, Z_raw, Wq, S, Z, N, K, group, 0, stream);
+}
+
+int w4a16_dequant_fmt(const void* Wq, const void* S, const void* Z, uint16_t* W16, int N, int K, int group, int flags,
+                      w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!flags_ok(flags)) return W4A16_ERR_SHAPE;
+    const bool sym = (flags & W4A16_FLAG_SYMMETRIC) != 0, bf = (flags & W4A16_FLAG_BF16) != 0;
+    if (!Wq || !S || !W16 || (!sym && !Z)) return W4A16_ERR_NULL;
+    int rc = check_weight_shape(N, K, group);
+    if (rc != W4A16_OK) return rc;
+    if (!aligned16(Wq) || !aligned16(S) || (!sym && !aligned16(Z)) || !aligned16(W16)) return W4A16_ERR_ALIGN;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != W4A16_OK) return rc;
+    if (!d->is_sm100) return W4A16_ERR_ARCH;
+    size_t words = (size_t)K * N / 8;
+    const uint32_t* z = sym ? nullptr : static_cast<const uint32_t*>(Z);
+    const unsigned blocks = (unsigned)((words + 255) / 256);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bf)
+        dequant_kernel<true><<<blocks, 256, 0, st>>>(static_cast<const uint32_t*>(Wq), static_cast<const uint16_t*>(S), z,
+                                                     W16, N, K / kGroup, kGroup / group, words);
+    else
+        dequant_kernel<false><<<blocks, 256, 0, st>>>(static_cast<const uint32_t*>(Wq), static_cast<const uint16_t*>(S), z,
+                                                      W16, N, K / kGroup, kGroup / group, words);
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
 int w4a16_dequant(const void* Wq, const void* S, const void* Z, uint16_t* W16, int N, int K, int group,
                   w4a16_stream_t stream) {
-    std::lock_guard<std::mutex> lock(g_mu);
-    if (!Wq || !S || !Z || !W16) return W4A16_ERR_NULL;
-    int rc = check_weight_shape(N, K, group);
-    if (rc != W4A16_OK) return rc;
-    if (!aligned16(Wq) || !aligned16(S) || !aligned16(Z) || !aligned16(W16)) return W4A16_ERR_ALIGN;
-    DeviceState* d = nullptr;
-    if ((rc = current_device(&d)) != W4A16_OK) return rc;
-    if (!d->is_sm100) return W4A16_ERR_ARCH;
-    size_t words = (size_t)K * N / 8;
-    dequant_kernel<<<(unsigned)((words + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint32_t*>(Wq), static_cast<const __half*>(S), static_cast<const uint32_t*>(Z),
-        reinterpret_cast<__half*>(W16), N, K / group, words);
-    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
+    if (!Z) return W4A16_ERR_NULL;
+    return w4a16_dequant_fmt(Wq, S, Z, W16, N, K, group, 0, stream);
 }
 
 }  // extern "C"
 
 namespace {
-// The body of w4a16_gemm_ex; the caller holds g_mu.
-int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
-                int group, int split_k, int path, w4a16_stream_t stream) {
-    if (!A || !Wq || !S || !Z || !C) return W4A16_ERR_NULL;
+
+// ---- kernel tables: one entry per template instantiation ------------------------------------------
+typedef void (*DecodeKernel)(const DecodeParams);
+template <int SG, bool BF>
+DecodeKernel decode_kernel_of(int mb, bool cluster) {
+    return cluster ? (mb == 2 ? gemm_decode_kernel<2, true, SG, BF> : gemm_decode_kernel<1, true, SG, BF>)
+                   : (mb == 2 ? gemm_decode_kernel<2, false, SG, BF> : gemm_decode_kernel<1, false, SG, BF>);
+}
+DecodeKernel decode_kernel(int mb, bool cluster, int sg, bool bf) {
+    if (bf) return sg == 1 ? decode_kernel_of<1, true>(mb, cluster) : sg == 2 ? decode_kernel_of<2, true>(mb, cluster)
+                                                                              : decode_kernel_of<4, true>(mb, cluster);
+    return sg == 1 ? decode_kernel_of<1, false>(mb, cluster) : sg == 2 ? decode_kernel_of<2, false>(mb, cluster)
+                                                                       : decode_kernel_of<4, false>(mb, cluster);
+}
+typedef void (*TileKernel)(const CUtensorMap, const TileParams);
+template <int SG, bool BF>
+TileKernel tile_kernel_of(int mt_index) {
+    return mt_index == 0 ? gemm_tile_kernel<16, SG, BF> : mt_index == 1 ? gemm_tile_kernel<32, SG, BF>
+         : mt_index == 2 ? gemm_tile_kernel<64, SG, BF> : mt_index == 3 ? gemm_tile_kernel<128, SG, BF>
+                                                                         : gemm_tile_kernel<256, SG, BF>;
+}
+TileKernel tile_kernel(int mt_index, int sg, bool bf) {
+    if (bf) return sg == 1 ? tile_kernel_of<1, true>(mt_index) : sg == 2 ? tile_kernel_of<2, true>(mt_index)
+                                                                         : tile_kernel_of<4, true>(mt_index);
+    return sg == 1 ? tile_kernel_of<1, false>(mt_index) : sg == 2 ? tile_kernel_of<2, false>(mt_index)
+                                                                  : tile_kernel_of<4, false>(mt_index);
+}
+
+// The body of every GEMM entry point; the caller holds g_mu.
+int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z, const uint16_t* bias, uint16_t* C,
+                int M, int N, int K, int group, int split_k, int path, int flags, int act, w4a16_stream_t stream) {
+    if (!flags_ok(flags)) return W4A16_ERR_SHAPE;
+    const bool sym = (flags & W4A16_FLAG_SYMMETRIC) != 0, bf = (flags & W4A16_FLAG_BF16) != 0;
+    if (!A || !Wq || !S || !C || (!sym && !Z)) return W4A16_ERR_NULL;
     int rc = check_weight_shape(N, K, group);
     if (rc != W4A16_OK) return rc;
     if (M < 1) return W4A16_ERR_SHAPE;
-    if (!aligned16(A) || !aligned16(Wq) || !aligned16(S) || !aligned16(Z) || !aligned16(C)) return W4A16_ERR_ALIGN;
-    const int G = K / group;
+    if (act < W4A16_ACT_NONE || act > W4A16_ACT_SILU) return W4A16_ERR_SHAPE;
+    if (!aligned16(A) || !aligned16(Wq) || !aligned16(S) || (!sym && !aligned16(Z)) || !aligned16(C))
+        return W4A16_ERR_ALIGN;
+    const int G = K / kGroup, sg = kGroup / group;
     if (split_k < 0 || split_k > G) return W4A16_ERR_SPLITK;
     if (path < W4A16_PATH_AUTO || path > W4A16_PATH_TILE) return W4A16_ERR_PATH;
     DeviceState* d = nullptr;
@@ -538,8 +595,10 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     path = resolve_path(M, N, G, split_k, d->sm_count, path, d->cluster_ok);
     if (split_k > 65535) return W4A16_ERR_SPLITK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const __half* Ah = reinterpret_cast<const __half*>(A);
-    __half* Ch = reinterpret_cast<__half*>(C);
+    const uint32_t* Zw = sym ? nullptr : static_cast<const uint32_t*>(Z);
+    Epilogue epi;
+    epi.bias = bias;
+    epi.act = act;
     // registered workspace: [16 KiB small-M tickets][128 KiB tile tickets][partial results]
     unsigned char* ws_body = d->ws ? static_cast<unsigned char*>(d->ws) + kWsFullHeaderBytes : nullptr;
     const size_t ws_body_bytes = d->ws_bytes > kWsFullHeaderBytes ? d->ws_bytes - kWsFullHeaderBytes : 0;
@@ -551,12 +610,20 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         if (mchunks > 65535) return W4A16_ERR_PATH;
         float* partials = reinterpret_cast<float*>(ws_body);
         dim3 grid(N / kTileN, mchunks, split_k);
-        gemm_simple_kernel<<<grid, 64, 0, st>>>(Ah, static_cast<const uint32_t*>(Wq), static_cast<const __half*>(S),
-                                                static_cast<const uint32_t*>(Z), Ch, partials, M, N, K, G, split_k);
+        if (bf)
+            gemm_simple_kernel<true><<<grid, 64, 0, st>>>(A, static_cast<const uint32_t*>(Wq),
+                                                          static_cast<const uint16_t*>(S), Zw, C, partials, M, N, K, G, sg,
+                                                          split_k, epi);
+        else
+            gemm_simple_kernel<false><<<grid, 64, 0, st>>>(A, static_cast<const uint32_t*>(Wq),
+                                                           static_cast<const uint16_t*>(S), Zw, C, partials, M, N, K, G, sg,
+                                                           split_k, epi);
         if (cudaGetLastError() != cudaSuccess) return W4A16_ERR_CUDA;
         if (split_k > 1) {
             size_t MN = (size_t)M * N;
-            splitk_reduce_kernel<<<(unsigned)((MN + 255) / 256), 256, 0, st>>>(partials, Ch, MN, split_k);
+            const unsigned blocks = (unsigned)((MN + 255) / 256);
+            if (bf) splitk_reduce_kernel<true><<<blocks, 256, 0, st>>>(partials, C, MN, N, split_k, epi);
+            else splitk_reduce_kernel<false><<<blocks, 256, 0, st>>>(partials, C, MN, N, split_k, epi);
             if (cudaGetLastError() != cudaSuccess) return W4A16_ERR_CUDA;
         }
         return W4A16_OK;
@@ -573,9 +640,9 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         if (!make_act_tensor_map(&tmap, A, M, K, g.mt)) return W4A16_ERR_CUDA;
         TileParams p;
         p.Wq = static_cast<const uint32_t*>(Wq);
-        p.S = static_cast<const __half*>(S);
-        p.Z = static_cast<const uint32_t*>(Z);
-        p.C = Ch;
+        p.S = static_cast<const uint16_t*>(S);
+        p.Z = Zw;
+        p.C = C;
         p.tickets = reinterpret_cast<int*>(d->ws ? static_cast<unsigned char*>(d->ws) + kWsHeaderBytes : nullptr);
         p.ws = reinterpret_cast<float*>(ws_body);
         p.M = M; p.N = N; p.K = K; p.G = G;
@@ -584,17 +651,16 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         p.split_k = g.split_k;
         p.nchunks = g.nchunks;
         p.stages = g.stages;
-        void (*kern)(const CUtensorMap, const TileParams) =
-            g.mt_index == 0 ? gemm_tile_kernel<16> : g.mt_index == 1 ? gemm_tile_kernel<32>
-            : g.mt_index == 2 ? gemm_tile_kernel<64> : g.mt_index == 3 ? gemm_tile_kernel<128>
-                                                                        : gemm_tile_kernel<256>;
-        if (!d->tile_attr_set[g.mt_index]) {
+        p.epi = epi;
+        TileKernel kern = tile_kernel(g.mt_index, sg, bf);
+        bool& attr_set = d->tile_attr_set[g.mt_index][log2_sg(sg)][bf ? 1 : 0];
+        if (!attr_set) {
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
                 cudaSuccess) {
                 cudaGetLastError();
                 return W4A16_ERR_CUDA;
             }
-            d->tile_attr_set[g.mt_index] = true;
+            attr_set = true;
         }
         // programmatic dependent launch: this kernel's prologue and weight prefetch may overlap the
         // tail of the previous kernel in the stream; it orders itself with griddepcontrol.wait
@@ -616,33 +682,33 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     }
 
     // W4A16_PATH_DECODE
-    DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, d->cluster_ok);
+    DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, d->cluster_ok, sg);
     if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
     if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
     // (the cluster exchange does not touch the workspace, but the contract stays the same for every schedule)
     if (g.split_k != 1 && ws_body_bytes < decode_partial_bytes(g)) return W4A16_ERR_WORKSPACE;
     DecodeParams p;
-    p.A = Ah;
+    p.A = A;
     p.Wq = static_cast<const uint32_t*>(Wq);
-    p.S = static_cast<const __half*>(S);
-    p.Z = static_cast<const uint32_t*>(Z);
-    p.C = Ch;
+    p.S = static_cast<const uint16_t*>(S);
+    p.Z = Zw;
+    p.C = C;
     p.ws = reinterpret_cast<float*>(ws_body);
     p.tickets = static_cast<int*>(d->ws);
     p.M = M; p.N = N; p.K = K; p.G = G; p.T = N / kTileN;
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    void (*kern)(const DecodeParams) =
-        g.cluster ? ((g.mb == 2) ? gemm_decode_kernel<2, 2, true> : gemm_decode_kernel<1, 2, true>)
-                  : ((g.mb == 2) ? gemm_decode_kernel<2, 2, false> : gemm_decode_kernel<1, 2, false>);
-    if (!d->decode_attr_set[g.mb][g.cps][g.cluster ? 1 : 0]) {
+    p.epi = epi;
+    DecodeKernel kern = decode_kernel(g.mb, g.cluster, sg, bf);
+    bool& attr_set = d->decode_attr_set[g.mb][g.cluster ? 1 : 0][log2_sg(sg)][bf ? 1 : 0];
+    if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
         }
-        d->decode_attr_set[g.mb][g.cps][g.cluster ? 1 : 0] = true;
+        attr_set = true;
     }
     // programmatic dependent launch (see the tile path above): prologue and weight prefetch may overlap
     // the tail of the previous kernel in the stream
@@ -673,7 +739,7 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
             // the device would not place the clusters: from now on the workspace exchange (and the path
             // rule that goes with it), starting with this call
             d->cluster_ok = false;
-            return gemm_locked(A, Wq, S, Z, C, M, N, K, group, split_k, path_asked, stream);
+            return gemm_locked(A, Wq, S, Z, bias, C, M, N, K, group, split_k, path_asked, flags, act, stream);
         }
         return W4A16_ERR_CUDA;
     }
@@ -683,10 +749,18 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
 
 extern "C" {
 
+int w4a16_gemm_fmt(const uint16_t* A, const void* Wq, const void* S, const void* Z, const uint16_t* bias, uint16_t* C,
+                   int M, int N, int K, int group, int split_k, int path, int flags, int act, w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (bias != nullptr && (reinterpret_cast<uintptr_t>(bias) & 1u)) return W4A16_ERR_ALIGN;
+    return gemm_locked(A, Wq, S, Z, bias, C, M, N, K, group, split_k, path, flags, act, stream);
+}
+
 int w4a16_gemm_ex(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
                   int group, int split_k, int path, w4a16_stream_t stream) {
     std::lock_guard<std::mutex> lock(g_mu);
-    return gemm_locked(A, Wq, S, Z, C, M, N, K, group, split_k, path, stream);
+    if (!Z) return W4A16_ERR_NULL;
+    return gemm_locked(A, Wq, S, Z, nullptr, C, M, N, K, group, split_k, path, 0, W4A16_ACT_NONE, stream);
 }
 
 int w4a16_gemm(const uint16_t* A, const void* Wq, const void* S, const void* Z, uint16_t* C, int M, int N, int K,
@@ -721,7 +795,7 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     if (rc != W4A16_OK) return rc;
     if (M < 1) return W4A16_ERR_SHAPE;
     if (!aligned16(A) || !aligned16(Wq) || !aligned16(S) || !aligned16(Z) || !aligned16(C)) return W4A16_ERR_ALIGN;
-    const int G = K / group;
+    const int G = K / kGroup, sg = kGroup / group;
     if (split_k < 0 || split_k > G) return W4A16_ERR_SPLITK;
     DeviceState* d = nullptr;
     if ((rc = current_device(&d)) != W4A16_OK) return rc;
@@ -729,7 +803,7 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return W4A16_ERR_CUDA;
 
-    const DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, false);   // no clusters here: this entry point keeps the path it was built with
+    const DecodeGeom g = decode_geom(M, N, G, split_k, d->sm_count, false, sg);   // no clusters here: this entry point keeps the path it was built with
     if (g.mchunks > 65535 || (long)g.mchunks * (N / kTileN) > kMaxTickets) return W4A16_ERR_PATH;
     if (g.smem_bytes > d->max_smem_optin) return W4A16_ERR_PATH;
     // the whole scratch need of this shape must fit the built-in array, or nothing is launched (a schedule of
@@ -754,25 +828,28 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
         return W4A16_ERR_CUDA;
     }
     DecodeParams p;
-    p.A = reinterpret_cast<const __half*>(A);
+    p.A = A;
     p.Wq = static_cast<const uint32_t*>(Wq);
-    p.S = static_cast<const __half*>(S);
+    p.S = static_cast<const uint16_t*>(S);
     p.Z = static_cast<const uint32_t*>(Z);
-    p.C = reinterpret_cast<__half*>(C);
+    p.C = C;
     p.ws = reinterpret_cast<float*>(ws + kWsHeaderBytes);
     p.tickets = reinterpret_cast<int*>(ws);
     p.M = M; p.N = N; p.K = K; p.G = G; p.T = N / kTileN;
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
-    auto kern = (g.mb == 2) ? gemm_decode_kernel<2, 2, false> : gemm_decode_kernel<1, 2, false>;
-    if (!d->decode_attr_set[g.mb][g.cps][0]) {
+    p.epi.bias = nullptr;
+    p.epi.act = kActNone;
+    DecodeKernel kern = decode_kernel(g.mb, false, sg, false);
+    bool& attr_set = d->decode_attr_set[g.mb][0][log2_sg(sg)][0];
+    if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
         }
-        d->decode_attr_set[g.mb][g.cps][0] = true;
+        attr_set = true;
     }
     kern<<<dim3(g.ctas, g.mchunks, 1), kDecThreads, g.smem_bytes, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;

@@ -27,15 +27,27 @@ namespace w4a16 {
 //         Inside a word, nibble p holds k offset 2 (p % 4) + p / 4, i.e. nibbles 0,4 = k+0,k+1;
 //         1,5 = k+2,k+3; 2,6 = k+4,k+5; 3,7 = k+6,k+7: the masks 0x000f000f / 0x00f000f0 on the
 //         word and on the word >> 8 then give four FP16x2 registers in ascending k.
-//   S   : 64 FP16 per block, element n % 64.
-//   Z   : 8 uint32 per block, word (n % 64) / 8, nibble n % 8.
+//   S   : per block, one row of 64 16-bit scales (FP16 or BF16 bit patterns) per quantization group
+//         inside the block: sg = 128 / group rows (group = 128, 64 or 32), row j = (k % 128) / group.
+//         Inside a row the scale of column c = n % 64 sits at position sz_perm(c): the four columns
+//         32 h + gq, + 8, + 16, + 24 that one lane of the warp-MMA kernel owns are neighbours (one
+//         64-bit shared load fetches the lane's four scales).
+//   Z   : the same rows and the same permutation, 4 bits per zero point (8 uint32 per row).  A
+//         symmetric format (zero point 8 for every weight) has no Z buffer at all.
 // ---------------------------------------------------------------------------------
-constexpr int kGroup = 128;
+constexpr int kGroup = 128;        // k per packed block (the scheduling unit); quantization groups divide it
 constexpr int kTileN = 64;
-constexpr int kBlockWords = 1024;  // uint32 per (tile, group) block of Wq
+constexpr int kBlockWords = 1024;  // uint32 per (tile, k-block) block of Wq
 constexpr int kBlockBytes = 4096;
-constexpr int kSBlockHalves = 64;
-constexpr int kZBlockWords = 8;
+constexpr int kSBlockHalves = 64;  // scales per row (one row per quantization group of the block)
+constexpr int kZBlockWords = 8;    // zero-point words per row
+constexpr int kSymZero = 8;        // zero point of the symmetric format (Eq. 1 with z fixed: q - 8 in -8 .. 7)
+
+// Position of column c (0..63) inside a row of scales / zero points.
+__host__ __device__ constexpr int sz_perm(int c) {
+    return (c & 32) + 4 * (c & 7) + 2 * ((c >> 4) & 1) + ((c >> 3) & 1);
+}
+__host__ __device__ constexpr bool group_ok(int group) { return group == 128 || group == 64 || group == 32; }
 
 // Word index inside a block of the word that holds column `col` (0..63) at k = 8*kw .. 8*kw+7
 // (kw = 0..15 inside the group).
@@ -160,54 +172,119 @@ __device__ __forceinline__ uint32_t lop3(uint32_t a, uint32_t b, uint32_t c) {
     return r;
 }
 
-// ------------------------------------------------------------------ nibble -> FP16
-// (w & 0x000f000f) | 0x64006400 is the FP16 pair (1024 + q_a, 1024 + q_b) for the nibbles
-// at bits 0..3 and 16..19;  (w & 0x00f000f0) | 0x64006400 is (1024 + 16 q_a, 1024 + 16 q_b)
-// for the nibbles at bits 4..7 and 20..23.  Both are exact FP16 values, so
-//   lo - (1024 + z)            = q - z   exactly (FP16 subtract of nearby integers)
-//   hi * (1/16) - (64 + z)     = q - z   exactly (FMA, the exact result is representable)
+// ------------------------------------------------------------------ nibble -> FP16 / BF16
+// Everything below works on 32-bit registers that hold two 16-bit floating-point values; the
+// template parameter BF selects BF16 (true) or FP16 (false) arithmetic.
+//
+// FP16 (ten fraction bits):
+//   (w & 0x000f000f) | 0x64006400 = (1024 + q_a, 1024 + q_b) for the nibbles at bits 0..3 / 16..19;
+//   (w & 0x00f000f0) | 0x54005400 = (  64 + q_a,   64 + q_b) for the nibbles at bits 4..7 / 20..23
+//   (the spacing of FP16 values at 64 is 1/16, so a nibble four bits up counts in units of one).
+//   Subtracting (1024 + z) resp. (64 + z) gives q - z exactly.
+// BF16 (seven fraction bits): a nibble fits the fraction only at bits 0..3, so the word is shifted by
+//   0, 4, 8, 12;  (w' & 0x000f000f) | 0x43004300 = (128 + q_a, 128 + q_b);  minus (128 + z) is exact.
+// Then ONE multiply by the scale in the same format: w16 = rn((q - z) * s), the single rounding of
+// Algorithm 1's "Dequantize to FP16" (resp. BF16).
 constexpr uint32_t kMaskLo = 0x000f000fu;
 constexpr uint32_t kMaskHi = 0x00f000f0u;
-constexpr uint32_t kMagic = 0x64006400u;  // FP16 1024.0 in both halves
+constexpr uint32_t kMagicLo = 0x64006400u;   // FP16 1024.0 twice
+constexpr uint32_t kMagicHi = 0x54005400u;   // FP16 64.0 twice
+constexpr uint32_t kMagicBf = 0x43004300u;   // BF16 128.0 twice
 constexpr int kLutAndOr = (0xF0 & 0xCC) | 0xAA;  // (a & b) | c
 
-// Eight weights of one column, ascending k, as four FP16 pairs.
-struct Half8 {
-    __half2 h[4];  // h[j] = (k + 2j, k + 2j + 1)
+template <bool BF>
+__device__ __forceinline__ uint32_t sub2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    if constexpr (BF) asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    else asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+template <bool BF>
+__device__ __forceinline__ uint32_t mul2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    if constexpr (BF) asm("mul.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    else asm("mul.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// The two per-column constants of the exact subtraction, both halves alike.
+//   FP16: lo = 1024 + z, hi = 64 + z;  BF16: lo = 128 + z (hi unused).
+template <bool BF>
+__device__ __forceinline__ uint32_t zconst_lo(uint32_t z) {
+    return BF ? (z * 0x00010001u + kMagicBf) : (z * 0x00010001u + kMagicLo);
+}
+template <bool BF>
+__device__ __forceinline__ uint32_t zconst_hi(uint32_t z) {
+    return BF ? 0u : (z * 0x00100010u + kMagicHi);
+}
+
+// Eight weights of one column, ascending k, as four register pairs: h[j] = (k + 2j, k + 2j + 1).
+struct Pack8 {
+    uint32_t h[4];
 };
 
-__device__ __forceinline__ __half2 u32_as_h2(uint32_t v) {
-    return *reinterpret_cast<__half2*>(&v);
-}
-__device__ __forceinline__ uint32_t h2_as_u32(__half2 v) {
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// zlo = FP16x2 (1024 + z) in both halves; zhi = FP16x2 -(64 + z) in both halves.
-__device__ __forceinline__ uint32_t zmagic_lo(uint32_t z) { return z * 0x00010001u + kMagic; }
-__device__ __forceinline__ uint32_t zmagic_hi(uint32_t z) { return z * 0x00100010u + 0xD400D400u; }
-
 // One packed word -> exact (q - z) for its eight k.
-__device__ __forceinline__ Half8 unpack_word(uint32_t w, __half2 zlo, __half2 zhi) {
-    const __half2 sixteenth = __float2half2_rn(0.0625f);
-    Half8 f;
-    const uint32_t w8 = w >> 8;
-    f.h[0] = __hsub2(u32_as_h2(lop3<kLutAndOr>(w, kMaskLo, kMagic)), zlo);
-    f.h[1] = __hfma2(u32_as_h2(lop3<kLutAndOr>(w, kMaskHi, kMagic)), sixteenth, zhi);
-    f.h[2] = __hsub2(u32_as_h2(lop3<kLutAndOr>(w8, kMaskLo, kMagic)), zlo);
-    f.h[3] = __hfma2(u32_as_h2(lop3<kLutAndOr>(w8, kMaskHi, kMagic)), sixteenth, zhi);
+template <bool BF>
+__device__ __forceinline__ Pack8 unpack_word(uint32_t w, uint32_t zlo, uint32_t zhi) {
+    Pack8 f;
+    if constexpr (BF) {
+        f.h[0] = sub2<true>(lop3<kLutAndOr>(w, kMaskLo, kMagicBf), zlo);
+        f.h[1] = sub2<true>(lop3<kLutAndOr>(w >> 4, kMaskLo, kMagicBf), zlo);
+        f.h[2] = sub2<true>(lop3<kLutAndOr>(w >> 8, kMaskLo, kMagicBf), zlo);
+        f.h[3] = sub2<true>(lop3<kLutAndOr>(w >> 12, kMaskLo, kMagicBf), zlo);
+    } else {
+        const uint32_t w8 = w >> 8;
+        f.h[0] = sub2<false>(lop3<kLutAndOr>(w, kMaskLo, kMagicLo), zlo);
+        f.h[1] = sub2<false>(lop3<kLutAndOr>(w, kMaskHi, kMagicHi), zhi);
+        f.h[2] = sub2<false>(lop3<kLutAndOr>(w8, kMaskLo, kMagicLo), zlo);
+        f.h[3] = sub2<false>(lop3<kLutAndOr>(w8, kMaskHi, kMagicHi), zhi);
+    }
     return f;
 }
 
-// One packed word -> w16 = fp16_rn((q - z) * s) for its eight k: exact (q - z), then one FP16
-// multiply by the column's scale (both halves of s2).  This is Algorithm 1's "Dequantize to
-// FP16": the multiplicand of the GEMM is the FP16-rounded weight, so every kernel that feeds
-// tensor cores goes through here.
-__device__ __forceinline__ Half8 dequant_word(uint32_t w, __half2 zlo, __half2 zhi, __half2 s2) {
-    Half8 f = unpack_word(w, zlo, zhi);
+// One packed word -> w16 = rn((q - z) * s) for its eight k (s2 = the column's scale in both halves).
+// Every kernel that feeds tensor cores goes through here: the multiplicand of the GEMM is the
+// weight rounded to the 16-bit format, as in Algorithm 1, Phase 1.
+template <bool BF>
+__device__ __forceinline__ Pack8 dequant_word(uint32_t w, uint32_t zlo, uint32_t zhi, uint32_t s2) {
+    Pack8 f = unpack_word<BF>(w, zlo, zhi);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) f.h[j] = __hmul2(f.h[j], s2);
+    for (int j = 0; j < 4; ++j) f.h[j] = mul2<BF>(f.h[j], s2);
     return f;
+}
+
+// FP32 -> 16-bit output, round to nearest even (the one cast of Algorithm 1, Phase 3).
+template <bool BF>
+__device__ __forceinline__ uint16_t cast_out(float v) {
+    uint16_t r;
+    if constexpr (BF) asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(v));
+    else asm("cvt.rn.f16.f32 %0, %1;" : "=h"(r) : "f"(v));
+    return r;
+}
+// Optional work fused into the final cast (none of it is in the paper's Algorithm 1; it stands for the
+// step that follows a linear layer): y = act(acc + bias[n]) in FP32, then the one rounding to 16 bits.
+constexpr int kActNone = 0, kActRelu = 1, kActSilu = 2;
+struct Epilogue {
+    const uint16_t* bias;   // [N] in the output's 16-bit format, or nullptr
+    int act;                // kActNone / kActRelu / kActSilu
+};
+
+// 16-bit value -> FP32 (exact).
+template <bool BF>
+__device__ __forceinline__ float widen(uint16_t v) {
+    if constexpr (BF) return __uint_as_float((uint32_t)v << 16);
+    float r;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(v));
+    return r;
+}
+
+// The final value of C[m, n] from its FP32 sum.
+template <bool BF>
+__device__ __forceinline__ uint16_t finish(float v, int n, const Epilogue& e) {
+    if (e.bias != nullptr) v += widen<BF>(e.bias[n]);
+    if (e.act == kActRelu) v = fmaxf(v, 0.f);
+    else if (e.act == kActSilu) v = v / (1.f + __expf(-v));
+    return cast_out<BF>(v);
 }
 
 }  // namespace w4a16

@@ -39,28 +39,32 @@ constexpr int kDecConsumers = kDecWarps * 32;
 constexpr int kDecThreads = kDecConsumers + 32;    // + producer warp
 constexpr int kDecMaxStages = 6;
 constexpr int kDecStageW = kDecUnitsPerStage * kBlockBytes;                 // 16384: nibbles
-constexpr int kDecStageS = kDecStageW;                                      // scales at 16384
-constexpr int kDecStageZ = kDecStageS + kDecUnitsPerStage * kSBlockHalves * 2;  // zeros at 16896
-constexpr int kDecStageA = 17152;                                           // activation rows
+constexpr int kDecStageS = kDecStageW;                                      // scale rows start here
 constexpr int kDecARowBytes = kDecUnitsPerStage * kGroup * 2 + 16;          // 1024 B of k + 16 B pad
 constexpr int kDecRedStride = 68;                  // floats per batch row in the reduce buffer
-constexpr int kDecUnitBytes = kBlockBytes + kSBlockHalves * 2 + kZBlockWords * 4;  // 4256
+// stage layout for SG scale rows per block: [4 x 4096 nibbles][4 x SG x 128 scales][4 x SG x 32 zeros][A rows]
+__host__ __device__ constexpr int dec_stage_z(int sg) { return kDecStageS + kDecUnitsPerStage * sg * kSBlockHalves * 2; }
+__host__ __device__ constexpr int dec_stage_a(int sg) { return dec_stage_z(sg) + kDecUnitsPerStage * sg * kZBlockWords * 4; }
+__host__ __device__ constexpr int dec_unit_bytes(int sg, bool sym) {
+    return kBlockBytes + sg * kSBlockHalves * 2 + (sym ? 0 : sg * kZBlockWords * 4);
+}
 
 struct DecodeParams {
-    const __half* A;
+    const uint16_t* A;
     const uint32_t* Wq;
-    const __half* S;
-    const uint32_t* Z;
-    __half* C;
+    const uint16_t* S;
+    const uint32_t* Z;  // nullptr: symmetric format, zero point 8
+    uint16_t* C;
     float* ws;          // partial tiles: [m chunk][2 * nchunks slots][8 MB rows][64] FP32
     int* tickets;       // zeroed counters: [m chunk][T]
-    int M, N, K, G, T;  // T = N / 64 column tiles
+    int M, N, K, G, T;  // G = K / 128 blocks along K, T = N / 64 column tiles
     int split_k;        // 0: balanced chunks; S >= 1: classic Split-K
     int nchunks;        // balanced: gridDim.x; classic: T * split_k
     int stages;
+    Epilogue epi;
 };
 
-__host__ __device__ inline int decode_stage_bytes(int mb) { return kDecStageA + 8 * mb * kDecARowBytes; }
+__host__ __device__ inline int decode_stage_bytes(int mb, int sg) { return dec_stage_a(sg) + 8 * mb * kDecARowBytes; }
 __host__ __device__ inline int decode_red_bytes(int mb) {
     return kDecUnitsPerStage * 8 * mb * kDecRedStride * 4;
 }
@@ -69,22 +73,85 @@ __host__ __device__ inline int decode_red_bytes(int mb) {
 // 6 everywhere: 6.5 against 6.0 us at K = 8192 / N = 2048, 18.8 against 9.2 with two batch blocks)
 constexpr int kDecMaxCluster = 6;
 __host__ __device__ inline int decode_xch_bytes(int mb, int slices) { return slices * 8 * mb * kTileN * 4; }
-__host__ __device__ inline int decode_smem_bytes(int mb, int stages, int cluster_slices) {
-    return 128 + decode_red_bytes(mb) + decode_xch_bytes(mb, cluster_slices) + stages * decode_stage_bytes(mb);
+__host__ __device__ inline int decode_smem_bytes(int mb, int sg, int stages, int cluster_slices) {
+    return 128 + decode_red_bytes(mb) + decode_xch_bytes(mb, cluster_slices) + stages * decode_stage_bytes(mb, sg);
 }
 
 // D += A . B with A = (a0: row gq, a1: row gq + 8, a2 / a3: the same rows, second k pair).
-__device__ __forceinline__ void mma_m16n8k16(float (&d)[4], __half2 a0, __half2 a1, __half2 a2, __half2 a3,
+template <bool BF>
+__device__ __forceinline__ void mma_m16n8k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                              uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(h2_as_u32(a0)), "r"(h2_as_u32(a1)), "r"(h2_as_u32(a2)), "r"(h2_as_u32(a3)), "r"(b0), "r"(b1));
+    if constexpr (BF)
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+            "{%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+            "{%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ void consumer_bar() {
     asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers) : "memory");
+}
+
+// Shared-memory loads at a 32-bit shared address plus a compile-time offset: the per-stage base
+// address is one register, everything else is an immediate.  (volatile + memory clobber keep them
+// after the barrier wait that guards the stage.)
+template <int OFF>
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2 + %3];" : "=r"(v.x), "=r"(v.y) : "r"(addr), "n"(OFF) : "memory");
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4 + %5];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(addr), "n"(OFF)
+                 : "memory");
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint32_t lds16(uint32_t addr) {
+    uint32_t v;
+    asm volatile("{\n\t.reg .b16 t;\n\tld.shared.u16 t, [%1 + %2];\n\tcvt.u32.u16 %0, t;\n\t}"
+                 : "=r"(v) : "r"(addr), "n"(OFF) : "memory");
+    return v;
+}
+
+// The producer's wait for a free ring slot.  It sleeps in the barrier unit between polls and is woken
+// by every barrier event of the CTA, so the poll loop is kept to a few instructions: the wall-clock
+// limit is checked only every 256th poll.
+__device__ __forceinline__ bool mbar_wait_producer(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity), "r"(100000u)
+            : "memory");
+        if (ok) return true;
+        if ((it & 255u) == 255u) {
+            unsigned long long t1;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+            if (t0 == 0) t0 = t1;
+            else if (t1 - t0 > kWaitLimitNs) break;
+        }
+    }
+    report_status(kStatusMbarTimeout);
+    return false;
 }
 
 // First unit of chunk i (i == nchunks gives the end of the last chunk).
@@ -131,27 +198,27 @@ struct DecStageIter {
     }
 };
 
-// MB = number of 8-row batch blocks one CTA handles (rows m0 .. m0 + 8 MB - 1).  CPS = CTAs the
-// launch wants resident per SM (2, or 3 with a two-stage ring and at most 72 registers: more warps
-// per scheduler pay on long launches, the shallower ring and the extra Split-K slices cost on short
-// ones; the host picks, see decode_geom).
+// MB = number of 8-row batch blocks one CTA handles (rows m0 .. m0 + 8 MB - 1); two CTAs per SM.
 // CL: the launch is made of thread-block clusters of split_k CTAs, one cluster per column tile and
 // one K slice per CTA (classic Split-K, every chunk on a CTA of its own).  The slices' partial tiles
 // then meet in the shared memory of the cluster's first CTA (distributed shared memory + one
 // hardware cluster barrier) instead of going through the workspace, a fence, a ticket and a reload:
 // Phase 3 of Algorithm 1 in about a tenth of the time, still summed in ascending K order.
-template <int MB, int CPS, bool CL>
-__global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const DecodeParams p) {
+// SG = scale / zero-point rows per 128-k block (quantization group 128 / SG); BF = BF16 arithmetic.
+template <int MB, bool CL, int SG, bool BF>
+__global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kRows = 8 * MB;
+    constexpr int kStageZ = dec_stage_z(SG), kStageA = dec_stage_a(SG);
+    constexpr int kStageBytes = kStageA + 8 * MB * kDecARowBytes;
+    const bool sym = p.Z == nullptr;
     const int mz = blockIdx.y;
     const int m0 = mz * kRows;
     const int rows = min(kRows, p.M - m0);  // batch rows this CTA really has
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = p.stages;
-    const int stage_bytes = decode_stage_bytes(MB);
 
-    // shared layout: [barriers + flag, 128 B][reduce buffer][stage 0][stage 1]...
+    // shared layout: [barriers + flag, 128 B][reduce buffer][exchange buffer (CL)][stage 0][stage 1]...
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);
     uint64_t* empty = full + kDecMaxStages;
     uint64_t* xbar = full + 2 * kDecMaxStages;   // CL only: the slices' partial tiles have landed (CTA 0's is used)
@@ -185,15 +252,17 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
 
     if (warp == kDecWarps) {
         // ------------------------------------------------ producer warp
+        const uint32_t unit_tx = (uint32_t)dec_unit_bytes(SG, sym);
         auto issue_weights = [&](const DecStageIter& it, unsigned char* st, uint64_t* bar, int gc) {
             bulk_g2s(st, p.Wq + (size_t)it.u * kBlockWords, (uint32_t)(gc * kBlockBytes), bar);
-            bulk_g2s(st + kDecStageS, p.S + (size_t)it.u * kSBlockHalves, (uint32_t)(gc * kSBlockHalves * 2), bar);
-            bulk_g2s(st + kDecStageZ, p.Z + (size_t)it.u * kZBlockWords, (uint32_t)(gc * kZBlockWords * 4), bar);
+            bulk_g2s(st + kDecStageS, p.S + (size_t)it.u * (SG * kSBlockHalves), (uint32_t)(gc * SG * kSBlockHalves * 2), bar);
+            if (!sym)
+                bulk_g2s(st + kStageZ, p.Z + (size_t)it.u * (SG * kZBlockWords), (uint32_t)(gc * SG * kZBlockWords * 4), bar);
         };
         auto issue_rows = [&](const DecStageIter& it, unsigned char* st, uint64_t* bar, int gc) {
-            const int g = it.group();  // the stage's units are groups g .. g + gc - 1 of tile t
+            const int g = it.group();  // the stage's units are blocks g .. g + gc - 1 of tile t
             for (int m = lane; m < rows; m += 32) {
-                bulk_g2s(st + kDecStageA + m * kDecARowBytes, p.A + (size_t)(m0 + m) * p.K + (size_t)g * kGroup,
+                bulk_g2s(st + kStageA + m * kDecARowBytes, p.A + (size_t)(m0 + m) * p.K + (size_t)g * kGroup,
                          (uint32_t)(gc * kGroup * 2), bar);
             }
         };
@@ -204,9 +273,9 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
                 if (lane == 0) {
                     const int gc = pre.units();
                     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full[i])),
-                                 "r"((uint32_t)(gc * kDecUnitBytes))
+                                 "r"((uint32_t)gc * unit_tx)
                                  : "memory");
-                    issue_weights(pre, stage0 + (size_t)i * stage_bytes, &full[i], gc);
+                    issue_weights(pre, stage0 + (size_t)i * kStageBytes, &full[i], gc);
                 }
             }
         }
@@ -216,15 +285,15 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
         uint32_t phase = 0;
         for (DecStageIter it(p); it.valid(); it.next(), ++n) {
             const int gc = it.units();
-            unsigned char* st = stage0 + (size_t)slot * stage_bytes;
+            unsigned char* st = stage0 + (size_t)slot * kStageBytes;
             if (n < stages) {
                 if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)(rows * gc * (kGroup * 2)));
                 __syncwarp();
                 issue_rows(it, st, &full[slot], gc);
             } else {
-                if (!mbar_wait(&empty[slot], phase ^ 1u)) return;  // status recorded
+                if (!mbar_wait_producer(&empty[slot], phase ^ 1u)) return;  // status recorded
                 if (lane == 0) {
-                    mbar_expect_tx(&full[slot], (uint32_t)(gc * kDecUnitBytes + rows * gc * (kGroup * 2)));
+                    mbar_expect_tx(&full[slot], (uint32_t)gc * unit_tx + (uint32_t)(rows * gc * (kGroup * 2)));
                     issue_weights(it, st, &full[slot], gc);
                 }
                 __syncwarp();
@@ -241,7 +310,8 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
     // ---------------------------------------------------- consumer warps
     const int gq = lane >> 2, tig = lane & 3;
     const int us = warp >> 1;         // which unit of the stage
-    const int r0 = (warp & 1) * 2;    // first of this warp's two 16-row sub-tiles
+    const int hh = warp & 1;          // which 32-column half of the tile: 16-column sub-tiles 2 hh, 2 hh + 1
+    const int r0 = hh * 2;
     float acc[2][MB][4];
 #pragma unroll
     for (int r = 0; r < 2; ++r)
@@ -250,12 +320,67 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[r][mb][i] = 0.f;
 
+    // Per-thread byte offsets inside a stage (everything else below is an immediate):
+    //   weights: this lane's 8 bytes of a column's 64-k line pair, k = 16 tig .. 16 tig + 15, of sub-tile 2 hh
+    //   activations: batch row gq, k = 16 tig ..
+    //   scales / zeros: the lane's four columns 32 hh + gq, + 8, + 16, + 24 are neighbours (sz_perm)
+    const uint32_t stage0_addr = smem_u32(stage0);
+    const uint32_t w_off = (uint32_t)(us * kBlockBytes + hh * 1024 + (tig >> 1) * 128 + ((gq + 4 * (tig >> 1)) & 7) * 16 + (tig & 1) * 8);
+    const uint32_t a_off = (uint32_t)(kStageA + us * (kGroup * 2) + gq * kDecARowBytes + tig * 32);
+    // SG = 4 (groups of 32 k): the lane's 16 k of a 64-k half lie in row 2 c + tig / 2
+    const int jlane = SG == 4 ? (tig >> 1) : 0;
+    const uint32_t s_off = (uint32_t)(kDecStageS + (us * SG + jlane) * (kSBlockHalves * 2) + (32 * hh + 4 * gq) * 2);
+    const uint32_t z_off = (uint32_t)(kStageZ + (us * SG + jlane) * (kZBlockWords * 4) + 16 * hh + 2 * gq);
+
+    // scale and zero-point constants of the lane's four columns (index 2 r + b: sub-tile r, column + 8 b)
+    uint32_t s2[4], zlo[4], zhi[4];
+    auto load_consts = [&](uint32_t st_addr, int j) {
+        const uint2 sv = (j == 0)   ? lds64<0>(st_addr + s_off)
+                         : (j == 1) ? lds64<kSBlockHalves * 2>(st_addr + s_off)
+                                    : lds64<2 * kSBlockHalves * 2>(st_addr + s_off);
+        s2[0] = __byte_perm(sv.x, 0, 0x1010);
+        s2[1] = __byte_perm(sv.x, 0, 0x3232);
+        s2[2] = __byte_perm(sv.y, 0, 0x1010);
+        s2[3] = __byte_perm(sv.y, 0, 0x3232);
+        if (sym) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                zlo[i] = zconst_lo<BF>(kSymZero);
+                zhi[i] = zconst_hi<BF>(kSymZero);
+            }
+        } else {
+            const uint32_t zz = (j == 0)   ? lds16<0>(st_addr + z_off)
+                                : (j == 1) ? lds16<kZBlockWords * 4>(st_addr + z_off)
+                                           : lds16<2 * kZBlockWords * 4>(st_addr + z_off);
+            const uint32_t t = zz * 0x00010001u;     // the four nibbles in both halves
+            const uint32_t t4 = t >> 4, t8 = t >> 8, t12 = t >> 12;
+            if constexpr (BF) {
+                zlo[0] = lop3<kLutAndOr>(t, kMaskLo, kMagicBf);
+                zlo[1] = lop3<kLutAndOr>(t4, kMaskLo, kMagicBf);
+                zlo[2] = lop3<kLutAndOr>(t8, kMaskLo, kMagicBf);
+                zlo[3] = lop3<kLutAndOr>(t12, kMaskLo, kMagicBf);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) zhi[i] = 0u;
+            } else {
+                zlo[0] = lop3<kLutAndOr>(t, kMaskLo, kMagicLo);
+                zlo[1] = lop3<kLutAndOr>(t4, kMaskLo, kMagicLo);
+                zlo[2] = lop3<kLutAndOr>(t8, kMaskLo, kMagicLo);
+                zlo[3] = lop3<kLutAndOr>(t12, kMaskLo, kMagicLo);
+                zhi[0] = lop3<kLutAndOr>(t << 4, kMaskHi, kMagicHi);
+                zhi[1] = lop3<kLutAndOr>(t, kMaskHi, kMagicHi);
+                zhi[2] = lop3<kLutAndOr>(t4, kMaskHi, kMagicHi);
+                zhi[3] = lop3<kLutAndOr>(t8, kMaskHi, kMagicHi);
+            }
+        }
+    };
+
     asm volatile("griddepcontrol.wait;" ::: "memory");
     float* const ws_mz = p.ws + (size_t)mz * (2 * (size_t)p.nchunks) * (kRows * kTileN);
     int* const tickets_mz = p.tickets + (size_t)mz * p.T;
 
     int slot = 0;
     uint32_t phase = 0;
+    uint32_t st_addr = stage0_addr;
     for (int ci = blockIdx.x; ci < p.nchunks; ci += gridDim.x) {
         const int u0 = chunk_begin(p, ci);
         const int u1 = chunk_begin(p, ci + 1);
@@ -268,55 +393,46 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
             const int gc = min(kDecUnitsPerStage, min(u1, tile_end) - u);
             if (!mbar_wait(&full[slot], phase)) return;  // status recorded; every consumer warp sees it
             if (us < gc) {
-                const unsigned char* st = stage0 + (size_t)slot * stage_bytes;
-                const unsigned char* wst = st + us * kBlockBytes;
-                const unsigned char* a_s = st + kDecStageA + us * (kGroup * 2);
-
-                // scales / zero points of this lane's columns 16 rr + gq and 16 rr + gq + 8, rr = r0, r0 + 1
-                const __half* sp = reinterpret_cast<const __half*>(st + kDecStageS + us * (kSBlockHalves * 2));
-                const uint4 zq = *reinterpret_cast<const uint4*>(st + kDecStageZ + us * (kZBlockWords * 4) + r0 * 8);
-                const uint32_t zw[4] = {zq.x, zq.y, zq.z, zq.w};   // columns 8 (2 r0 + i) .. + 7
-                __half2 s_a[2], s_b[2], zlo_a[2], zhi_a[2], zlo_b[2], zhi_b[2];
-#pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    s_a[r] = __half2half2(sp[(r0 + r) * 16 + gq]);
-                    s_b[r] = __half2half2(sp[(r0 + r) * 16 + gq + 8]);
-                    const uint32_t za = (zw[2 * r] >> (4 * gq)) & 15u, zb = (zw[2 * r + 1] >> (4 * gq)) & 15u;
-                    zlo_a[r] = u32_as_h2(zmagic_lo(za));
-                    zhi_a[r] = u32_as_h2(zmagic_hi(za));
-                    zlo_b[r] = u32_as_h2(zmagic_lo(zb));
-                    zhi_b[r] = u32_as_h2(zmagic_hi(zb));
-                }
-                // this lane's 8 bytes of a column's 64-k line pair: k = 16 tig .. 16 tig + 15
-                const int woff = (tig >> 1) * 128 + ((gq + 4 * (tig >> 1)) & 7) * 16 + (tig & 1) * 8;
+                const uint32_t wa = st_addr + w_off, aa = st_addr + a_off;
+                if constexpr (SG == 1) load_consts(st_addr, 0);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
+                    if constexpr (SG == 2) load_consts(st_addr, c);
+                    if constexpr (SG == 4) load_consts(st_addr, 2 * c);
                     // B fragments: batch row 8 mb + gq, 16 consecutive k per lane
                     uint32_t bw[MB][8];
 #pragma unroll
                     for (int mb = 0; mb < MB; ++mb) {
-                        const uint4* ap =
-                            reinterpret_cast<const uint4*>(a_s + (mb * 8 + gq) * kDecARowBytes + c * 128 + tig * 32);
-                        const uint4 x = ap[0], y = ap[1];
+                        uint4 x, y;
+                        if (c == 0) {
+                            x = mb == 0 ? lds128<0>(aa) : lds128<8 * kDecARowBytes>(aa);
+                            y = mb == 0 ? lds128<16>(aa) : lds128<8 * kDecARowBytes + 16>(aa);
+                        } else {
+                            x = mb == 0 ? lds128<128>(aa) : lds128<8 * kDecARowBytes + 128>(aa);
+                            y = mb == 0 ? lds128<128 + 16>(aa) : lds128<8 * kDecARowBytes + 128 + 16>(aa);
+                        }
                         bw[mb][0] = x.x; bw[mb][1] = x.y; bw[mb][2] = x.z; bw[mb][3] = x.w;
                         bw[mb][4] = y.x; bw[mb][5] = y.y; bw[mb][6] = y.z; bw[mb][7] = y.w;
                     }
 #pragma unroll
                     for (int r = 0; r < 2; ++r) {
-                        const unsigned char* sub = wst + (c * 8 + 2 * (r0 + r)) * 256 + woff;
-                        const uint2 wa = *reinterpret_cast<const uint2*>(sub);        // column 16 rr + gq
-                        const uint2 wb = *reinterpret_cast<const uint2*>(sub + 256);  // column 16 rr + gq + 8
-                        const uint32_t wwa[2] = {wa.x, wa.y}, wwb[2] = {wb.x, wb.y};
+                        // sub-block (c, 2 (2 hh + r)) holds columns 16 rr + gq, the next one columns + 8
+                        uint2 va, vb;
+                        if (c == 0 && r == 0) { va = lds64<0>(wa); vb = lds64<256>(wa); }
+                        else if (c == 0)      { va = lds64<512>(wa); vb = lds64<512 + 256>(wa); }
+                        else if (r == 0)      { va = lds64<2048>(wa); vb = lds64<2048 + 256>(wa); }
+                        else                  { va = lds64<2048 + 512>(wa); vb = lds64<2048 + 512 + 256>(wa); }
+                        const uint32_t wwa[2] = {va.x, va.y}, wwb[2] = {vb.x, vb.y};
 #pragma unroll
                         for (int wi = 0; wi < 2; ++wi) {
-                            const Half8 fa = dequant_word(wwa[wi], zlo_a[r], zhi_a[r], s_a[r]);
-                            const Half8 fb = dequant_word(wwb[wi], zlo_b[r], zhi_b[r], s_b[r]);
+                            const Pack8 fa = dequant_word<BF>(wwa[wi], zlo[2 * r], zhi[2 * r], s2[2 * r]);
+                            const Pack8 fb = dequant_word<BF>(wwb[wi], zlo[2 * r + 1], zhi[2 * r + 1], s2[2 * r + 1]);
 #pragma unroll
                             for (int mb = 0; mb < MB; ++mb) {
-                                mma_m16n8k16(acc[r][mb], fa.h[0], fb.h[0], fa.h[1], fb.h[1], bw[mb][4 * wi],
-                                             bw[mb][4 * wi + 1]);
-                                mma_m16n8k16(acc[r][mb], fa.h[2], fb.h[2], fa.h[3], fb.h[3], bw[mb][4 * wi + 2],
-                                             bw[mb][4 * wi + 3]);
+                                mma_m16n8k16<BF>(acc[r][mb], fa.h[0], fb.h[0], fa.h[1], fb.h[1], bw[mb][4 * wi],
+                                                 bw[mb][4 * wi + 1]);
+                                mma_m16n8k16<BF>(acc[r][mb], fa.h[2], fb.h[2], fa.h[3], fb.h[3], bw[mb][4 * wi + 2],
+                                                 bw[mb][4 * wi + 3]);
                             }
                         }
                     }
@@ -324,9 +440,11 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[slot]);
+            st_addr += (uint32_t)kStageBytes;
             if (++slot == stages) {
                 slot = 0;
                 phase ^= 1u;
+                st_addr = stage0_addr;
             }
             u += gc;
             if (u != tile_end && u != u1) continue;
@@ -373,7 +491,7 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
                         const int n = idx & (kTileN - 1), m = idx >> 6;
                         float v = xch[idx];
                         for (int sl = 1; sl < p.split_k; ++sl) v += xch[sl * (kRows * kTileN) + idx];
-                        p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
+                        p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = finish<BF>(v, t * kTileN + n, p.epi);
                     }
                 }
                 return;   // one slice per CTA: nothing follows
@@ -384,7 +502,7 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
 #pragma unroll
                 for (int w = 1; w < kDecUnitsPerStage; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
                 if (whole)
-                    p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
+                    p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = finish<BF>(v, t * kTileN + n, p.epi);
                 else
                     my_slot[idx] = v;
             }
@@ -424,7 +542,7 @@ __global__ void __launch_bounds__(kDecThreads, CPS) gemm_decode_kernel(const Dec
                             c += 2;
                         }
                         if (c <= c_last) v += __ldcg(src + (size_t)c * cstride);
-                        p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = __float2half_rn(v);
+                        p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = finish<BF>(v, t * kTileN + n, p.epi);
                     }
                 }
             }

@@ -91,9 +91,9 @@ __host__ __device__ constexpr int tile_stage_bytes(int mt) { return mt * tile_st
 
 struct TileParams {
     const uint32_t* Wq;
-    const __half* S;
-    const uint32_t* Z;
-    __half* C;
+    const uint16_t* S;
+    const uint32_t* Z;   // nullptr: symmetric format, zero point 8
+    uint16_t* C;
     float* ws;       // partial tiles: [2 * nchunks slots][MT][128] FP32
     int* tickets;    // zeroed counters: [tile][16 epilogue warps]
     int M, N, K, G;
@@ -102,6 +102,7 @@ struct TileParams {
     int split_k;     // 0: balanced chunks; S >= 1: classic Split-K
     int nchunks;
     int stages;
+    Epilogue epi;
 };
 
 // ------------------------------------------------------------------ tcgen05 / TMA wrappers
@@ -199,9 +200,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
     return d;
 }
 
-// kind::f16 instruction descriptor: FP32 accumulator, FP16 A and B, both K-major, M = 128, N = mt.
-__host__ __device__ constexpr uint32_t tile_idesc(int mt) {
-    return (1u << 4) | ((uint32_t)(mt >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
+// kind::f16 instruction descriptor: FP32 accumulator, A and B both FP16 or both BF16, both K-major,
+// M = 128, N = mt.
+__host__ __device__ constexpr uint32_t tile_idesc(int mt, bool bf) {
+    return (1u << 4) | (bf ? ((1u << 7) | (1u << 10)) : 0u) | ((uint32_t)(mt >> 3) << 17) |
+           ((uint32_t)(kTileCols >> 4) << 24);
 }
 
 // ------------------------------------------------------------------ chunk schedule
@@ -305,15 +308,18 @@ __device__ __forceinline__ bool wait_slot_free(uint64_t* retired, const RingPos&
     return mbar_wait(retired + (t & 1u) * kTileMaxStages + r.slot, (t >> 1) & 1u);
 }
 
-// Packed words, scale and zero point of one thread's column for one stage of 32 * NW k.
-template <int NW>
+// Packed words, scales and zero points of one thread's column for one stage of 32 * NW k (NR
+// quantization groups).
+template <int NW, int NR>
 struct StageRegs {
-    uint4 w[NW];      // w[i]: k = 32 i .. 32 i + 31 of the stage
-    uint32_t s;       // FP16 scale bits
-    uint32_t zw;      // zero-point word of the column's 8-column block
+    uint4 w[NW];        // w[i]: k = 32 i .. 32 i + 31 of the stage
+    uint32_t s[NR];     // 16-bit scale patterns
+    uint32_t zw[NR];    // zero-point words that hold the column's nibble
 };
 
-template <int MT>
+// MT = batch rows per tile; SG = scale / zero-point rows per 128-k block (quantization group 128 / SG);
+// BF = BF16 instead of FP16 activations, scales, weights and output.
+template <int MT, int SG, bool BF>
 __global__ void __launch_bounds__(tile_threads(MT), 1)
 gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -321,7 +327,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     // dynamic segment starts
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kStageBytes = tile_stage_bytes(MT);
-    constexpr uint32_t kIdesc = tile_idesc(MT);
+    constexpr uint32_t kIdesc = tile_idesc(MT, BF);
     constexpr int kCW = MT / kTileSets;                  // accumulator columns (batch rows) per epilogue warp
     constexpr int kNI = tile_issuers(MT);                // MMA-issuing warps, one accumulator (set) each
     constexpr int kDBufs = tile_dbufs(MT);               // accumulators per issuer: accumulator (b, i) sits
@@ -332,6 +338,8 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
     constexpr int kACol = tile_a_col_base(MT);
     constexpr int kNW = kStageK / 32;                    // 16-byte chunks of a thread's column per stage
     constexpr int kPF = tile_prefetch(MT);
+    constexpr int kNR = SG / kSPU > 0 ? SG / kSPU : 1;   // scale rows one stage touches
+    const bool sym = p.Z == nullptr;
 
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [R]  activation box landed AND operand stored in TMEM
     uint64_t* retired = full + kTileMaxStages;                   // [2][R]  the stage's MMAs retired: slot free
@@ -461,7 +469,8 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         // word offsets of this thread's two 16-byte chunks inside a block's 64-k half
         const int wo0 = (col >> 3) * 64 + (col & 7) * 4;
         const int wo1 = (col >> 3) * 64 + 32 + (((col & 7) + 4) & 7) * 4;
-        const int zsh = 4 * (col & 7);
+        const int zp = sz_perm(col);         // position of this column's scale / zero point inside a row
+        const int zsh = 4 * (zp & 7);
 
         // this set's first stage inside a segment
         auto first_own = [&](const SegWalk& w) { return (int)(((uint32_t)set - w.n0) & 3u); };
@@ -472,7 +481,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         int jl = 0;
         bool l_in = false;                      // this thread's column exists (not past the matrix edge)
         const uint32_t* lw = nullptr;           // the stage's first word of this thread's 8-column block
-        const unsigned short* ls = nullptr;
+        const uint16_t* ls = nullptr;
         const uint32_t* lz = nullptr;
         auto point = [&]() {                    // cursor entered a new segment: settle on a stage, set pointers
             while (wl.valid()) {
@@ -485,11 +494,13 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             l_in = t64 * kTileN < p.N;
             const size_t blk = (size_t)t64 * p.G + (wl.g0 + jl / kSPU);
             lw = p.Wq + blk * kBlockWords + (jl % kSPU) * 512;
-            ls = reinterpret_cast<const unsigned short*>(p.S) + blk * kSBlockHalves + col;
-            lz = p.Z + blk * kZBlockWords + (col >> 3);
+            // first scale row of the stage: a 64-k stage of a block with SG >= 2 rows starts at row (SG / 2) * half
+            const size_t row = blk * SG + (SG >= kSPU ? (jl % kSPU) * (SG / kSPU) : 0);
+            ls = p.S + row * kSBlockHalves + zp;
+            lz = sym ? nullptr : p.Z + row * kZBlockWords + (zp >> 3);
         };
         // load the cursor's stage (zeros past the matrix edge) and advance the cursor
-        auto fetch = [&](StageRegs<kNW>& r) {
+        auto fetch = [&](StageRegs<kNW, kNR>& r) {
             if (!wl.valid()) return;
             if (l_in) {
 #pragma unroll
@@ -497,19 +508,22 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
                     r.w[2 * h] = __ldg(reinterpret_cast<const uint4*>(lw + h * 512 + wo0));
                     r.w[2 * h + 1] = __ldg(reinterpret_cast<const uint4*>(lw + h * 512 + wo1));
                 }
-                r.s = __ldg(ls);
-                r.zw = __ldg(lz);
+#pragma unroll
+                for (int i = 0; i < kNR; ++i) {
+                    r.s[i] = __ldg(ls + i * kSBlockHalves);
+                    r.zw[i] = sym ? 0u : __ldg(lz + i * kZBlockWords);
+                }
             } else {
 #pragma unroll
                 for (int i = 0; i < kNW; ++i) r.w[i] = make_uint4(0, 0, 0, 0);
-                r.s = 0;
-                r.zw = 0;
+#pragma unroll
+                for (int i = 0; i < kNR; ++i) { r.s[i] = 0; r.zw[i] = 0; }
             }
             jl += kTileSets;
             if (jl < wl.stages_in_seg()) {
                 lw += (kTileSets / kSPU) * kBlockWords;
-                ls += (kTileSets / kSPU) * kSBlockHalves;
-                lz += (kTileSets / kSPU) * kZBlockWords;
+                ls += (kTileSets / kSPU) * (SG * kSBlockHalves);
+                if (!sym) lz += (kTileSets / kSPU) * (SG * kZBlockWords);
             } else {
                 wl.next();
                 point();
@@ -518,7 +532,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         point();
         // register ring of prefetched stages, written out so that no slot is ever copied
         static_assert(kPF == 2 || kPF == 3, "the ring below has two or three slots");
-        StageRegs<kNW> pf0, pf1, pf2;
+        StageRegs<kNW, kNR> pf0, pf1, pf2;
         fetch(pf0);
         fetch(pf1);
         if (kPF == 3) fetch(pf2);
@@ -532,10 +546,15 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
         RingPos rp{0, 0u, 0u};
         bool ok = true;
         // one stage of this thread's column -> kSlotCols TMEM columns of the ring slot
-        auto convert = [&](const StageRegs<kNW>& cur, uint32_t n) -> bool {
-            const uint32_t z = (cur.zw >> zsh) & 15u;
-            const __half2 s2 = u32_as_h2(cur.s * 0x00010001u);
-            const __half2 zlo = u32_as_h2(zmagic_lo(z)), zhi = u32_as_h2(zmagic_hi(z));
+        auto convert = [&](const StageRegs<kNW, kNR>& cur, uint32_t n) -> bool {
+            uint32_t s2[kNR], zlo[kNR], zhi[kNR];
+#pragma unroll
+            for (int i = 0; i < kNR; ++i) {
+                const uint32_t z = sym ? (uint32_t)kSymZero : ((cur.zw[i] >> zsh) & 15u);
+                s2[i] = cur.s[i] * 0x00010001u;
+                zlo[i] = zconst_lo<BF>(z);
+                zhi[i] = zconst_hi<BF>(z);
+            }
             // the MMAs that read this slot one ring turn ago must have retired
             if (rp.turn != 0u && !wait_slot_free(retired, rp)) return false;
             tc_fence_after();
@@ -543,12 +562,14 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll
             for (int c = 0; c < kNW; ++c) {      // 32 k -> 16 TMEM columns at a time
                 const uint32_t ww[4] = {cur.w[c].x, cur.w[c].y, cur.w[c].z, cur.w[c].w};
+                constexpr int kRowDiv = 4 / SG > 0 ? 4 / SG : 1;   // 32-k chunks per scale row (group / 32)
+                const int ri = (c / kRowDiv) < kNR ? (c / kRowDiv) : kNR - 1;
                 uint32_t regs[16];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const Half8 f = dequant_word(ww[i], zlo, zhi, s2);
+                    const Pack8 f = dequant_word<BF>(ww[i], zlo[ri], zhi[ri], s2[ri]);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) regs[4 * i + q] = h2_as_u32(f.h[q]);
+                    for (int q = 0; q < 4; ++q) regs[4 * i + q] = f.h[q];
                 }
                 tc_st16(a_t + 16 * c, regs);
             }
@@ -623,7 +644,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll
                         for (int q = 0; q < kStep; ++q) {
                             const int m = m_base + cc + q;
-                            if (m < p.M) p.C[(size_t)m * p.N + n] = __float2half_rn(__uint_as_float(v[q]));
+                            if (m < p.M) p.C[(size_t)m * p.N + n] = finish<BF>(__uint_as_float(v[q]), n, p.epi);
                         }
                     }
                 } else {
@@ -689,7 +710,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
 #pragma unroll
                             for (int q = 0; q < kStep; ++q) {
                                 const int m = m_base + m0 + q;
-                                if (m < p.M) p.C[(size_t)m * p.N + n] = __float2half_rn(acc[q]);
+                                if (m < p.M) p.C[(size_t)m * p.N + n] = finish<BF>(acc[q], n, p.epi);
                             }
                         }
                     }

@@ -7,7 +7,7 @@
 namespace w4a16 {
 
 // ------------------------------------------------------------------ pack
-// Decode a packed word's position: idx -> block, column inside the tile, first k inside the group.
+// Decode a packed word's position: idx -> block, column inside the tile, first k inside the block.
 __device__ __forceinline__ void word_position(size_t idx, size_t& blk, int& col, int& kw) {
     const int within = (int)(idx & 1023);
     blk = idx >> 10;
@@ -36,36 +36,55 @@ __global__ void pack_wq_kernel(const uint32_t* __restrict__ raw, uint32_t* __res
     out[idx] = w;
 }
 
-__global__ void pack_s_kernel(const uint16_t* __restrict__ raw, uint16_t* __restrict__ out, int N, int G,
+// Scales: packed position idx = ((blk * sg + j) * 64 + sz_perm(col)); one thread per raw scale.
+__global__ void pack_s_kernel(const uint16_t* __restrict__ raw, uint16_t* __restrict__ out, int N, int G, int sg,
                               size_t total) {
-    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // over (t, g, j, col)
     if (idx >= total) return;
     const int col = (int)(idx & 63);
-    const size_t blk = idx >> 6;
+    const size_t row = idx >> 6;                 // (t * G + g) * sg + j
+    const int j = (int)(row % sg);
+    const size_t blk = row / sg;
     const int t = (int)(blk / G), g = (int)(blk % G);
-    out[idx] = raw[(size_t)g * N + (size_t)t * kTileN + col];
+    out[row * kSBlockHalves + sz_perm(col)] = raw[(size_t)(g * sg + j) * N + (size_t)t * kTileN + col];
 }
 
-__global__ void pack_z_kernel(const uint8_t* __restrict__ raw, uint32_t* __restrict__ out, int N, int G,
+// Zero points: one thread per packed word (eight permuted positions of one row).
+__global__ void pack_z_kernel(const uint8_t* __restrict__ raw, uint32_t* __restrict__ out, int N, int G, int sg,
                               size_t total_words) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total_words) return;
-    const int rb = (int)(idx & 7);
-    const size_t blk = idx >> 3;
+    const int wi = (int)(idx & 7);
+    const size_t row = idx >> 3;
+    const int j = (int)(row % sg);
+    const size_t blk = row / sg;
     const int t = (int)(blk / G), g = (int)(blk % G);
     uint32_t w = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        w |= (uint32_t)(raw[(size_t)g * N + (size_t)t * kTileN + rb * 8 + i] & 15u) << (4 * i);
+    for (int col = 0; col < kTileN; ++col) {
+        const int p = sz_perm(col);
+        if ((p >> 3) == wi)
+            w |= (uint32_t)(raw[(size_t)(g * sg + j) * N + (size_t)t * kTileN + col] & 15u) << (4 * (p & 7));
+    }
     out[idx] = w;
 }
 
+// Scale (16-bit pattern) and zero point of column `col` for the k-word kw (0..15) of block blk.
+__device__ __forceinline__ void load_sz(const uint16_t* __restrict__ S, const uint32_t* __restrict__ Z, size_t blk,
+                                        int sg, int col, int kw, uint16_t& s, uint32_t& z) {
+    const int j = (kw * 8) / (kGroup / sg);
+    const size_t row = blk * sg + j;
+    const int p = sz_perm(col);
+    s = S[row * kSBlockHalves + p];
+    z = Z == nullptr ? (uint32_t)kSymZero : ((Z[row * kZBlockWords + (p >> 3)] >> (4 * (p & 7))) & 15u);
+}
+
 // ------------------------------------------------------------------ dequant
-// Algorithm 1, Phase 1 as a standalone kernel: one thread per packed word, eight FP16
-// results w16 = fp16_rn((q - z) * s): (q - z) is formed exactly in FP16 and multiplied by s
-// with one FP16 multiply (round-to-nearest-even, subnormals kept).
-__global__ void dequant_kernel(const uint32_t* __restrict__ Wq, const __half* __restrict__ S,
-                               const uint32_t* __restrict__ Z, __half* __restrict__ W16, int N, int G,
+// Algorithm 1, Phase 1 as a standalone kernel: one thread per packed word, eight results
+// w16 = rn((q - z) * s) in the 16-bit format: (q - z) is formed exactly and multiplied by s with one
+// multiply (round-to-nearest-even, subnormals kept).  Z == nullptr: symmetric format, z = 8.
+template <bool BF>
+__global__ void dequant_kernel(const uint32_t* __restrict__ Wq, const uint16_t* __restrict__ S,
+                               const uint32_t* __restrict__ Z, uint16_t* __restrict__ W16, int N, int G, int sg,
                                size_t total_words) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total_words) return;
@@ -73,21 +92,22 @@ __global__ void dequant_kernel(const uint32_t* __restrict__ Wq, const __half* __
     int col, kw;
     word_position(idx, blk, col, kw);
     const int t = (int)(blk / G), g = (int)(blk % G);
-    const uint32_t z = (Z[blk * kZBlockWords + (col >> 3)] >> (4 * (col & 7))) & 15u;
-    const __half s = S[blk * kSBlockHalves + col];
-    const Half8 f = dequant_word(Wq[idx], u32_as_h2(zmagic_lo(z)), u32_as_h2(zmagic_hi(z)), __half2half2(s));
-    __half* p = W16 + (size_t)(g * kGroup + kw * 8) * N + (size_t)t * kTileN + col;
+    uint16_t s;
+    uint32_t z;
+    load_sz(S, Z, blk, sg, col, kw, s, z);
+    const Pack8 f = dequant_word<BF>(Wq[idx], zconst_lo<BF>(z), zconst_hi<BF>(z), (uint32_t)s * 0x00010001u);
+    uint16_t* p = W16 + (size_t)(g * kGroup + kw * 8) * N + (size_t)t * kTileN + col;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        p[(size_t)(2 * j) * N] = __low2half(f.h[j]);
-        p[(size_t)(2 * j + 1) * N] = __high2half(f.h[j]);
+        p[(size_t)(2 * j) * N] = (uint16_t)(f.h[j] & 0xffffu);
+        p[(size_t)(2 * j + 1) * N] = (uint16_t)(f.h[j] >> 16);
     }
 }
 
 // ------------------------------------------------------------------ plain GEMM
 // Correct-first kernel: one thread per output column of a 64-column tile, kSimpleMB batch
 // rows per thread, FP32 FMA over this CTA's K-slice.  Grid: (N/64,
-// ceil(M/kSimpleMB), split_k).  With split_k == 1 it writes FP16 C, else FP32 partials
+// ceil(M/kSimpleMB), split_k).  With split_k == 1 it writes C, else FP32 partials
 // ws[split][M][N] (Algorithm 1, Phase 2) for splitk_reduce_kernel.
 constexpr int kSimpleMB = 4;
 
@@ -97,10 +117,11 @@ __device__ __forceinline__ void slice_of(int G, int split_k, int sp, int& g0, in
     ng = base + (sp < rem ? 1 : 0);
 }
 
+template <bool BF>
 __global__ void __launch_bounds__(64)
-gemm_simple_kernel(const __half* __restrict__ A, const uint32_t* __restrict__ Wq, const __half* __restrict__ S,
-                   const uint32_t* __restrict__ Z, __half* __restrict__ C, float* __restrict__ ws, int M, int N,
-                   int K, int G, int split_k) {
+gemm_simple_kernel(const uint16_t* __restrict__ A, const uint32_t* __restrict__ Wq, const uint16_t* __restrict__ S,
+                   const uint32_t* __restrict__ Z, uint16_t* __restrict__ C, float* __restrict__ ws, int M, int N,
+                   int K, int G, int sg, int split_k, Epilogue epi) {
     const int t = blockIdx.x, m0 = blockIdx.y * kSimpleMB, sp = blockIdx.z;
     const int col = threadIdx.x;  // column inside the tile
     int g0, ng;
@@ -112,21 +133,24 @@ gemm_simple_kernel(const __half* __restrict__ A, const uint32_t* __restrict__ Wq
 
     for (int g = g0; g < g0 + ng; ++g) {
         const size_t blk = (size_t)t * G + g;
-        const int z = (int)((Z[blk * kZBlockWords + (col >> 3)] >> (4 * (col & 7))) & 15u);
-        const float s = __half2float(S[blk * kSBlockHalves + col]);
         const uint32_t* wb = Wq + blk * kBlockWords;
         for (int kw = 0; kw < kGroup / 8; ++kw) {
+            uint16_t sb;
+            uint32_t z;
+            load_sz(S, Z, blk, sg, col, kw, sb, z);
+            const float s = widen<BF>(sb);
             const uint32_t w = wb[block_word_index(col, kw)];
             const int k0 = g * kGroup + kw * 8;
 #pragma unroll
             for (int p = 0; p < 8; ++p) {
                 const int off = 2 * (p & 3) + (p >> 2);
                 const int q = (int)((w >> (4 * p)) & 15u);
-                const float w16 = __half2float(__float2half_rn((float)(q - z) * s));
+                // (q - z) * s is exact in FP32; one rounding to the 16-bit format, as in Phase 1
+                const float w16 = widen<BF>(cast_out<BF>((float)(q - (int)z) * s));
 #pragma unroll
                 for (int mm = 0; mm < kSimpleMB; ++mm) {
                     if (m0 + mm < M)
-                        acc[mm] = fmaf(__half2float(A[(size_t)(m0 + mm) * K + k0 + off]), w16, acc[mm]);
+                        acc[mm] = fmaf(widen<BF>(A[(size_t)(m0 + mm) * K + k0 + off]), w16, acc[mm]);
                 }
             }
         }
@@ -136,21 +160,22 @@ gemm_simple_kernel(const __half* __restrict__ A, const uint32_t* __restrict__ Wq
     for (int mm = 0; mm < kSimpleMB; ++mm) {
         if (m0 + mm < M) {
             if (split_k == 1)
-                C[(size_t)(m0 + mm) * N + n] = __float2half_rn(acc[mm]);
+                C[(size_t)(m0 + mm) * N + n] = finish<BF>(acc[mm], n, epi);
             else
                 ws[((size_t)sp * M + m0 + mm) * N + n] = acc[mm];
         }
     }
 }
 
-// Algorithm 1, Phase 3: C = fp16_rn(sum_{i<S} C_i), ascending i, FP32.
-__global__ void splitk_reduce_kernel(const float* __restrict__ ws, __half* __restrict__ C, size_t MN,
-                                     int split_k) {
+// Algorithm 1, Phase 3: C = rn16(sum_{i<S} C_i), ascending i, FP32.
+template <bool BF>
+__global__ void splitk_reduce_kernel(const float* __restrict__ ws, uint16_t* __restrict__ C, size_t MN, int N,
+                                     int split_k, Epilogue epi) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= MN) return;
     float acc = ws[i];
     for (int s = 1; s < split_k; ++s) acc += ws[(size_t)s * MN + i];
-    C[i] = __float2half_rn(acc);
+    C[i] = finish<BF>(acc, (int)(i % (size_t)N), epi);
 }
 
 // Diagnostic: one warp waits on a barrier that nobody ever arrives on, with a limit of `limit_ns`.  The wait

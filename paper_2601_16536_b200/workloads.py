@@ -75,20 +75,38 @@ def _f16_bits(x: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(x.astype(np.float16)).view(np.uint16)
 
 
-def draw_weights(K: int, N: int, seed: int, group: int = GROUP) -> Dict[str, np.ndarray]:
-    """Wq, S, Z in the raw layout: q uniform 0..15, s ~ U[0.002, 0.02], z uniform 0..15."""
+def _bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Storage format of the drawn numbers only: float32 -> the nearest BF16 pattern (ties to even)."""
+    b = np.ascontiguousarray(x.astype(np.float32)).view(np.uint32).astype(np.uint64)
+    return ((b + 0x7FFF + ((b >> 16) & 1)) >> 16).astype(np.uint16)
+
+
+def _bits16(x: np.ndarray, bf16: bool) -> np.ndarray:
+    return _bf16_bits(x) if bf16 else _f16_bits(x)
+
+
+SYM_ZERO = 8    # the zero point every weight of a symmetric format has
+
+
+def draw_weights(K: int, N: int, seed: int, group: int = GROUP, symmetric: bool = False,
+                 bf16: bool = False) -> Dict[str, np.ndarray]:
+    """Wq, S, Z in the raw layout: q uniform 0..15, s ~ U[0.002, 0.02], z uniform 0..15 (all 8 for a
+    symmetric format: the array is what a checker needs, the symmetric GPU path takes no Z at all).
+    ``bf16`` stores the scales as BF16 instead of FP16 patterns."""
     G = K // group
     rq = np.random.Generator(np.random.PCG64([seed, 1]))
     rs = np.random.Generator(np.random.PCG64([seed, 2]))
     rz = np.random.Generator(np.random.PCG64([seed, 3]))
     Wq = rq.integers(0, 2 ** 32, size=(K // 8, N), dtype=np.uint64).astype(np.uint32)
-    S = _f16_bits(rs.uniform(0.002, 0.02, size=(G, N)).astype(np.float32))
+    S = _bits16(rs.uniform(0.002, 0.02, size=(G, N)).astype(np.float32), bf16)
     Z = rz.integers(0, 16, size=(G, N), dtype=np.uint8)
+    if symmetric:
+        Z = np.full((G, N), SYM_ZERO, dtype=np.uint8)
     return {"Wq": Wq, "S": S, "Z": Z}
 
 
 def draw_activations(M: int, K: int, seed: int, sigma: float = 1.0,
-                     outliers: bool = False) -> np.ndarray:
+                     outliers: bool = False, bf16: bool = False) -> np.ndarray:
     """A ~ N(0, sigma); with ``outliers`` round(0.01 K) seeded columns are scaled x20."""
     ra = np.random.Generator(np.random.PCG64([seed, 0]))
     A = ra.standard_normal(size=(M, K), dtype=np.float32) * np.float32(sigma)
@@ -96,7 +114,7 @@ def draw_activations(M: int, K: int, seed: int, sigma: float = 1.0,
         ro = np.random.Generator(np.random.PCG64([seed, 4]))
         cols = ro.permutation(K)[: int(round(0.01 * K))]
         A[:, cols] *= np.float32(20.0)
-    return _f16_bits(A)
+    return _bits16(A, bf16)
 
 
 def make_case(case: Case, group: int = GROUP) -> Dict[str, np.ndarray]:
@@ -106,14 +124,16 @@ def make_case(case: Case, group: int = GROUP) -> Dict[str, np.ndarray]:
 
 
 def make_problem(M: int, K: int, N: int, seed: int, group: int = GROUP,
-                 sigma: float = 1.0, outliers: bool = False) -> Dict[str, np.ndarray]:
-    d = draw_weights(K, N, seed, group)
-    d["A"] = draw_activations(M, K, seed, sigma, outliers)
+                 sigma: float = 1.0, outliers: bool = False, symmetric: bool = False,
+                 bf16: bool = False) -> Dict[str, np.ndarray]:
+    d = draw_weights(K, N, seed, group, symmetric, bf16)
+    d["A"] = draw_activations(M, K, seed, sigma, outliers, bf16)
     return d
 
 
 def make_exact_problem(M: int, K: int, N: int, seed: int, group: int = GROUP,
-                       e_lo: int = -8, e_hi: int = -4) -> Dict[str, np.ndarray]:
+                       e_lo: int = -8, e_hi: int = -4, symmetric: bool = False,
+                       bf16: bool = False) -> Dict[str, np.ndarray]:
     """Inputs for which every product and partial sum is exactly representable:
     A in {-1, 0, 1}, scales 2**E with integer E in [e_lo, e_hi].
     Returns the raw arrays plus ``A_int`` (int8) and ``E`` (int8)."""
@@ -123,15 +143,17 @@ def make_exact_problem(M: int, K: int, N: int, seed: int, group: int = GROUP,
     E = r.integers(e_lo, e_hi + 1, size=(G, N), dtype=np.int8)
     Wq = r.integers(0, 2 ** 32, size=(K // 8, N), dtype=np.uint64).astype(np.uint32)
     Z = r.integers(0, 16, size=(G, N), dtype=np.uint8)
-    S = _f16_bits(np.ldexp(np.float32(1.0), E.astype(np.int32)).astype(np.float32))
-    A = _f16_bits(A_int.astype(np.float32))
+    if symmetric:
+        Z = np.full((G, N), SYM_ZERO, dtype=np.uint8)
+    S = _bits16(np.ldexp(np.float32(1.0), E.astype(np.int32)).astype(np.float32), bf16)
+    A = _bits16(A_int.astype(np.float32), bf16)
     return {"A": A, "A_int": A_int, "Wq": Wq, "S": S, "Z": Z, "E": E}
 
 
-def algorithmic_bytes(M: int, K: int, N: int, group: int = GROUP) -> int:
-    """Bytes one call must move: packed weights + FP16 scales + 4-bit zeros + A + C."""
+def algorithmic_bytes(M: int, K: int, N: int, group: int = GROUP, symmetric: bool = False) -> int:
+    """Bytes one call must move: packed weights + 16-bit scales + 4-bit zeros (none when symmetric) + A + C."""
     G = K // group
-    return K * N // 2 + G * N * 2 + G * N // 2 + 2 * M * K + 2 * M * N
+    return K * N // 2 + G * N * 2 + (0 if symmetric else G * N // 2) + 2 * M * K + 2 * M * N
 
 
 def iter_cases(configs=(1, 2, 3, 4, 5)) -> Iterator[Case]:

@@ -40,7 +40,12 @@ def test_packed_sizes_hold_exactly_the_raw_information(lib):
     # unsupported shapes report size 0
     assert lib.w4a16_packed_wq_bytes(100, 4096, 128) == 0
     assert lib.w4a16_packed_wq_bytes(4096, 4000, 128) == 0
-    assert lib.w4a16_packed_wq_bytes(4096, 4096, 64) == 0
+    assert lib.w4a16_packed_wq_bytes(4096, 4096, 48) == 0
+    # smaller quantization groups: the same nibbles, proportionally more scales and zero points
+    for group in (32, 64):
+        assert lib.w4a16_packed_wq_bytes(4096, 4096, group) == 4096 * 4096 // 2
+        assert lib.w4a16_packed_s_bytes(4096, 4096, group) == (4096 // group) * 4096 * 2
+        assert lib.w4a16_packed_z_bytes(4096, 4096, group) == (4096 // group) * 4096 // 2
 
 
 def test_choose_split_k_is_always_acceptable(lib):
@@ -99,7 +104,7 @@ def test_argument_errors_are_reported_before_any_device_work(lib):
     p = (p + 15) // 16 * 16
     assert lib.w4a16_gemm(None, p, p, p, p, 1, 64, 128, 128, 1, None) == -1
     assert lib.w4a16_gemm(p, p, p, p, None, 1, 64, 128, 128, 1, None) == -1
-    assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 128, 64, 1, None) == -2      # group
+    assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 128, 48, 1, None) == -2      # group
     assert lib.w4a16_gemm(p, p, p, p, p, 1, 60, 128, 128, 1, None) == -2     # N % 64
     assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 100, 128, 1, None) == -2     # K % 128
     assert lib.w4a16_gemm(p, p, p, p, p, 0, 64, 128, 128, 1, None) == -2     # M
@@ -108,7 +113,15 @@ def test_argument_errors_are_reported_before_any_device_work(lib):
     assert lib.w4a16_gemm(p, p, p, p, p, 1, 64, 128, 128, -1, None) == -4
     assert lib.w4a16_gemm_ex(p, p, p, p, p, 1, 64, 128, 128, 1, 9, None) == -9
     assert lib.w4a16_pack(None, p, p, p, p, p, 64, 128, 128, None) == -1
-    assert lib.w4a16_pack(p, p, p, p, p, p, 64, 128, 32, None) == -2
+    assert lib.w4a16_pack(p, p, p, p, p, p, 64, 128, 16, None) == -2
+    assert lib.w4a16_pack(p, p, None, p, p, p, 64, 128, 128, None) == -1      # the plain entry points need Z
+    assert lib.w4a16_gemm(p, p, p, None, p, 1, 64, 128, 128, 1, None) == -1
+    assert lib.w4a16_pack_fmt(p, p, None, p, p, None, 64, 128, 128, 0, None) == -1   # asymmetric: Z required
+    assert lib.w4a16_pack_fmt(p, p, None, p, p, None, 64, 128, 128, 8, None) == -2   # unknown flag
+    assert lib.w4a16_gemm_fmt(p, p, p, None, None, p, 1, 64, 128, 128, 1, 0, 0, 0, None) == -1
+    assert lib.w4a16_gemm_fmt(p, p, p, p, None, p, 1, 64, 128, 128, 1, 0, 0, 7, None) == -2   # unknown activation
+    assert lib.w4a16_gemm_fmt(p, p, p, p, p + 1, p, 1, 64, 128, 128, 1, 0, 0, 0, None) == -3  # odd bias address
+    assert lib.w4a16_dequant_fmt(p, p, None, p, 64, 128, 128, 0, None) == -1
     assert lib.w4a16_dequant(p, p, p, None, 64, 128, 128, None) == -1
     assert lib.w4a16_dequant(p, p, p, p + 4, 64, 128, 128, None) == -3
     assert lib.w4a16_gemm_host(None, p, p, p, p, p, p, 1, 64, 128, 128, 1, None) == -1

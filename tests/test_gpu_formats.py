@@ -1,0 +1,124 @@
+"""GPU parity of the format variants through the C ABI (w4a16_pack_fmt / w4a16_dequant_fmt /
+w4a16_gemm_fmt): quantization groups of 32 and 64 along K, the symmetric case of Eq. 1 (zero point 8,
+no Z buffer), BF16 instead of FP16 (Section 1 names both as the dequantization target), and the fused
+bias / activation step.  Dequantization is compared bit for bit, products within the GEMM tolerances,
+exactly representable inputs bit for bit on every path and split."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_16536_b200 import binding as B
+from paper_2601_16536_b200 import workloads as wl
+from gpu_util import assert_close, ensure_ws, to_dev
+
+pytestmark = pytest.mark.gpu
+
+PATHS = {"simple": B.PATH_SIMPLE, "decode": B.PATH_DECODE, "tile": B.PATH_TILE}
+
+
+def _flags(symmetric, bf16=False):
+    return (B.FLAG_SYMMETRIC if symmetric else 0) | (B.FLAG_BF16 if bf16 else 0)
+
+
+def _dev16(bits, bf16=False):
+    t = torch.from_numpy(bits.view(np.int16)).cuda()
+    return t.view(torch.bfloat16 if bf16 else torch.float16)
+
+
+def _pack(d, N, K, group, symmetric, bf16=False):
+    return B.w4a16_pack(to_dev(d["Wq"]), _dev16(d["S"], bf16), None if symmetric else to_dev(d["Z"]), N, K, group,
+                        _flags(symmetric, bf16))
+
+
+def _bits(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _f64(t):
+    return t.to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("group", [32, 64, 128])
+@pytest.mark.parametrize("symmetric", [False, True])
+def test_dequant_is_bit_exact(group, symmetric):
+    K, N = 640, 192      # five k-blocks, three column tiles
+    d = wl.draw_weights(K, N, seed=800 + group, group=group, symmetric=symmetric)
+    # scales over the whole FP16 range, subnormal and huge ones among them
+    r = np.random.Generator(np.random.PCG64(group))
+    d["S"] = r.integers(0, 0x7C00, size=d["S"].shape, dtype=np.uint64).astype(np.uint16)
+    pw = _pack(d, N, K, group, symmetric)
+    assert (pw.Z is None) == symmetric
+    got = _bits(B.w4a16_dequant(pw))
+    want = oracle.dequant(d["Wq"], d["S"], d["Z"], K, N, group)
+    assert np.array_equal(got, want)
+
+
+SHAPES = [(1, 640, 192), (5, 1152, 128), (16, 896, 256), (40, 768, 128)]
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("group,symmetric", [(32, False), (64, False), (128, True), (32, True), (64, True)])
+@pytest.mark.parametrize("M,K,N", SHAPES)
+def test_gemm_matches_oracle(path, group, symmetric, M, K, N):
+    d = wl.make_problem(M, K, N, seed=M + K + group, group=group, symmetric=symmetric)
+    pw = _pack(d, N, K, group, symmetric)
+    ws = ensure_ws(M, N, K, (0, 1, 2, 3))
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, group)
+    for split_k in (0, 1, 3):
+        C = B.w4a16_gemm(_dev16(d["A"]), pw, split_k=split_k, path=PATHS[path])
+        torch.cuda.synchronize()
+        assert B.w4a16_device_status() == 0
+        assert_close(_f64(C), ref, "%s g%d sym%d M%d split %d" % (path, group, symmetric, M, split_k))
+    del ws
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("group,symmetric", [(32, False), (64, True), (128, True)])
+def test_exact_inputs_are_bit_equal(path, group, symmetric):
+    M, K, N = 7, 1152, 128
+    d = wl.make_exact_problem(M, K, N, seed=31 + group, group=group, symmetric=symmetric)
+    pw = _pack(d, N, K, group, symmetric)
+    want = oracle.gemm_int(d["A_int"], d["Wq"], d["E"], d["Z"], M, N, K, group)
+    ws = ensure_ws(M, N, K, (0, 1, 2, 4, 9))
+    for split_k in (0, 1, 2, 4, 9):
+        C = B.w4a16_gemm(_dev16(d["A"]), pw, split_k=split_k, path=PATHS[path])
+        torch.cuda.synchronize()
+        assert np.array_equal(_bits(C), want), "split_k=%d" % split_k
+    del ws
+
+
+@pytest.mark.parametrize("group,symmetric", [(32, False), (64, False), (128, True)])
+def test_full_size_decode_shape_whole_output(group, symmetric):
+    # the benchmark's decode shape with the format variants, automatic path and split, whole C
+    M, K, N = 8, 11008, 4096
+    d = wl.make_problem(M, K, N, seed=group, group=group, symmetric=symmetric)
+    pw = _pack(d, N, K, group, symmetric)
+    ws = ensure_ws(M, N, K, 0)
+    C = B.w4a16_gemm(_dev16(d["A"]), pw)
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    assert_close(_f64(C), oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, group), "g%d sym%d" % (group, symmetric))
+    del ws
+
+
+@pytest.mark.parametrize("path,M", [("simple", 3), ("decode", 6), ("decode", 16), ("tile", 24), ("tile", 200)])
+@pytest.mark.parametrize("act", ["none", "relu", "silu"])
+def test_bias_and_activation_are_applied_before_the_final_rounding(path, M, act):
+    K, N = 1152, 256
+    d = wl.make_problem(M, K, N, seed=M * 7 + len(act))
+    pw = _pack(d, N, K, 128, False)
+    r = np.random.Generator(np.random.PCG64(M))
+    bias_bits = r.standard_normal(N).astype(np.float16).view(np.uint16)
+    bias = bias_bits.view(np.float16).astype(np.float64)
+    ws = ensure_ws(M, N, K, (0, 1, 3))
+    ref = oracle.epilogue(oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128), bias, act)
+    code = {"none": B.ACT_NONE, "relu": B.ACT_RELU, "silu": B.ACT_SILU}[act]
+    for split_k in (0, 1, 3):
+        C = B.w4a16_gemm(_dev16(d["A"]), pw, split_k=split_k, path=PATHS[path], bias=_dev16(bias_bits), act=code)
+        torch.cuda.synchronize()
+        assert B.w4a16_device_status() == 0
+        assert_close(_f64(C), ref, "%s M%d %s split %d" % (path, M, act, split_k))
+        if act == "relu":
+            assert np.all(_f64(C) >= 0)
+    del ws
