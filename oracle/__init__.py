@@ -58,6 +58,16 @@ def lib():
         L.orc_gemm_kslice.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp]
         L.orc_gemm_int.restype = i
         L.orc_gemm_int.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
+        L.orc_bf16_to_f32.restype = ctypes.c_float
+        L.orc_bf16_to_f32.argtypes = [ctypes.c_uint16]
+        L.orc_f64_to_bf16_rn.restype = ctypes.c_uint16
+        L.orc_f64_to_bf16_rn.argtypes = [ctypes.c_double]
+        L.orc_dequant_fmt.restype = None
+        L.orc_dequant_fmt.argtypes = [vp, vp, vp, i, i, i, i, vp]
+        L.orc_gemm_fmt.restype = None
+        L.orc_gemm_fmt.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.orc_gemm_int_fmt.restype = i
+        L.orc_gemm_int_fmt.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp]
         L.orc_num_threads.restype = i
         L.orc_num_threads.argtypes = []
         _lib = L
@@ -85,6 +95,14 @@ def f64_to_f16_rn(x: float) -> int:
     return int(lib().orc_f64_to_f16_rn(float(x)))
 
 
+def bf16_to_f32(bits: int) -> float:
+    return float(lib().orc_bf16_to_f32(int(bits) & 0xFFFF))
+
+
+def f64_to_bf16_rn(x: float) -> int:
+    return int(lib().orc_f64_to_bf16_rn(float(x)))
+
+
 def unpack(Wq: np.ndarray, K: int, N: int) -> np.ndarray:
     """q[k, n] (uint8, [K, N]) from the raw words Wq uint32 [K/8, N]."""
     Wq = _chk(Wq, np.uint32, (K // 8, N))
@@ -93,24 +111,34 @@ def unpack(Wq: np.ndarray, K: int, N: int) -> np.ndarray:
     return q
 
 
-def dequant(Wq, S, Z, K: int, N: int, group: int = 128) -> np.ndarray:
-    """FP16 bit patterns (uint16, [K, N]) of fp16_rn((q - z) * s)."""
+def dequant(Wq, S, Z, K: int, N: int, group: int = 128, bf16: bool = False) -> np.ndarray:
+    """16-bit patterns (uint16, [K, N]) of rn16((q - z) * s); FP16, or BF16 with ``bf16``."""
     Wq = _chk(Wq, np.uint32, (K // 8, N))
     S = _chk(S, np.uint16, (K // group, N))
     Z = _chk(Z, np.uint8, (K // group, N))
     W16 = np.empty((K, N), dtype=np.uint16)
-    lib().orc_dequant(_p(Wq), _p(S), _p(Z), K, N, group, _p(W16))
+    if bf16:
+        lib().orc_dequant_fmt(_p(Wq), _p(S), _p(Z), K, N, group, 1, _p(W16))
+    else:
+        lib().orc_dequant(_p(Wq), _p(S), _p(Z), K, N, group, _p(W16))
     return W16
 
 
-def gemm(A, Wq, S, Z, M: int, N: int, K: int, group: int = 128, cols=None) -> np.ndarray:
+def gemm(A, Wq, S, Z, M: int, N: int, K: int, group: int = 128, cols=None, bf16: bool = False) -> np.ndarray:
     """C_ref (float64, [M, N]) = sum_k A[m,k] * w16[k,n] in FP64.
 
-    ``cols=(n0, n1)`` computes only those columns (the rest are NaN)."""
+    ``cols=(n0, n1)`` computes only those columns (the rest are NaN); ``bf16``: A, S and the
+    dequantized weights are BF16 instead of FP16."""
     A = _chk(A, np.uint16, (M, K))
     Wq = _chk(Wq, np.uint32, (K // 8, N))
     S = _chk(S, np.uint16, (K // group, N))
     Z = _chk(Z, np.uint8, (K // group, N))
+    if bf16:
+        if cols is not None:
+            raise ValueError("cols is not available for the BF16 format")
+        C = np.empty((M, N), dtype=np.float64)
+        lib().orc_gemm_fmt(_p(A), _p(Wq), _p(S), _p(Z), M, N, K, group, 1, _p(C))
+        return C
     if cols is None:
         C = np.empty((M, N), dtype=np.float64)
         lib().orc_gemm(_p(A), _p(Wq), _p(S), _p(Z), M, N, K, group, _p(C))
@@ -132,14 +160,14 @@ def gemm_kslice(A, Wq, S, Z, M, N, K, group, k0, k1) -> np.ndarray:
     return C
 
 
-def gemm_int(A_int, Wq, E, Z, M, N, K, group=128) -> np.ndarray:
-    """Exact case: integer A (int8), scales 2**E (int8 exponents); FP16 bits [M, N]."""
+def gemm_int(A_int, Wq, E, Z, M, N, K, group=128, bf16: bool = False) -> np.ndarray:
+    """Exact case: integer A (int8), scales 2**E (int8 exponents); FP16 (or BF16) bits [M, N]."""
     A_int = _chk(A_int, np.int8, (M, K))
     Wq = _chk(Wq, np.uint32, (K // 8, N))
     E = _chk(E, np.int8, (K // group, N))
     Z = _chk(Z, np.uint8, (K // group, N))
     C = np.empty((M, N), dtype=np.uint16)
-    rc = lib().orc_gemm_int(_p(A_int), _p(Wq), _p(E), _p(Z), M, N, K, group, _p(C))
+    rc = lib().orc_gemm_int_fmt(_p(A_int), _p(Wq), _p(E), _p(Z), M, N, K, group, 1 if bf16 else 0, _p(C))
     if rc != 0:
         raise ValueError("exponent range too wide for the exact oracle")
     return C

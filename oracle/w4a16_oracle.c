@@ -90,6 +90,63 @@ uint16_t orc_f64_to_f16_rn(double x)
 
 uint16_t orc_f32_to_f16_rn(float x) { return orc_f64_to_f16_rn((double)x); }
 
+/* ---- bfloat16 <-> binary32/64 (Section 1 names BF16 beside FP16 as the dequantization target) ----
+ * bfloat16: 1 sign, 8 exponent (bias 127), 7 fraction bits: the upper half of a binary32. */
+float orc_bf16_to_f32(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) & 1u;
+    int      e    = (int)((h >> 7) & 0xFFu);
+    uint32_t f    = (uint32_t)(h & 0x7Fu);
+    double v;
+    if (e == 0) {
+        v = ldexp((double)f, -133);              /* subnormal or zero: f * 2^-133 */
+    } else if (e == 255) {
+        v = f ? NAN : INFINITY;
+    } else {
+        v = ldexp((double)(128u + f), e - 134);  /* (1 + f/128) * 2^(e-127) */
+    }
+    return (float)(sign ? -v : v);
+}
+
+/* Round a double to the nearest bfloat16, ties to even; overflow -> Inf. */
+uint16_t orc_f64_to_bf16_rn(double x)
+{
+    uint16_t sign = 0;
+    if (isnan(x)) return 0x7FC0u;
+    if (signbit(x)) { sign = 0x8000u; x = -x; }
+    if (isinf(x)) return (uint16_t)(sign | 0x7F80u);
+    if (x == 0.0) return sign;
+    int ex;
+    (void)frexp(x, &ex);
+    int e = ex - 1;                               /* floor(log2 x) */
+    /* spacing of bfloat16 values around x: 2^(e-7) for normals, 2^-133 below 2^-126 */
+    int ulp_exp = (e < -126) ? -133 : (e - 7);
+    double r = nearbyint(ldexp(x, -ulp_exp));     /* integer count of ulps, ties to even */
+    if (r == 0.0) return sign;
+    double v = ldexp(r, ulp_exp);
+    if (v >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7F80u);   /* rounded past the largest finite value */
+    int ev;
+    (void)frexp(v, &ev);
+    int fe = ev - 1;
+    if (fe < -126) {
+        uint32_t frac = (uint32_t)ldexp(v, 133);
+        return (uint16_t)(sign | frac);
+    } else {
+        uint32_t mant = (uint32_t)ldexp(v, 7 - fe);            /* in [128, 256) */
+        return (uint16_t)(sign | ((uint32_t)(fe + 127) << 7) | (mant - 128u));
+    }
+}
+
+/* The 16-bit format of activations, scales, dequantized weights and output: 0 = FP16, 1 = BF16. */
+static inline double orc_widen(uint16_t bits, int bf16)
+{
+    return (double)(bf16 ? orc_bf16_to_f32(bits) : orc_f16_to_f32(bits));
+}
+static inline uint16_t orc_round16(double x, int bf16)
+{
+    return bf16 ? orc_f64_to_bf16_rn(x) : orc_f64_to_f16_rn(x);
+}
+
 /* ---- unpack (Section 2.2: INT4 values packed into INT32 words) ---- */
 
 /* q[k, n] for all k < K, n < N as one byte each, row-major [K, N]. */
@@ -109,23 +166,29 @@ static inline int orc_q_at(const uint32_t *Wq, int N, int k, int n)
 
 /* ---- Dequant(W) = s (W - z), rounded once to FP16 (Eq. 2; Algorithm 1, Phase 1) ---- */
 
-static inline uint16_t orc_dequant_one(int q, int z, uint16_t s_bits)
+static inline uint16_t orc_dequant_one(int q, int z, uint16_t s_bits, int bf16)
 {
-    double s = (double)orc_f16_to_f32(s_bits);
-    return orc_f64_to_f16_rn((double)(q - z) * s);   /* subtract first, multiply once */
+    double s = orc_widen(s_bits, bf16);
+    return orc_round16((double)(q - z) * s, bf16);   /* subtract first, multiply once, round once */
 }
 
-/* W16[k, n], FP16 bits, row-major [K, N]. */
-void orc_dequant(const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
-                 int K, int N, int group, uint16_t *W16)
+/* W16[k, n], 16-bit patterns (FP16, or BF16 when bf16 != 0), row-major [K, N]. */
+void orc_dequant_fmt(const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                     int K, int N, int group, int bf16, uint16_t *W16)
 {
     #pragma omp parallel for schedule(static)
     for (int k = 0; k < K; ++k) {
         int g = k / group;
         for (int n = 0; n < N; ++n)
             W16[(size_t)k * N + n] =
-                orc_dequant_one(orc_q_at(Wq, N, k, n), Z[(size_t)g * N + n], S[(size_t)g * N + n]);
+                orc_dequant_one(orc_q_at(Wq, N, k, n), Z[(size_t)g * N + n], S[(size_t)g * N + n], bf16);
     }
+}
+
+void orc_dequant(const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                 int K, int N, int group, uint16_t *W16)
+{
+    orc_dequant_fmt(Wq, S, Z, K, N, group, 0, W16);
 }
 
 /* ---- C = A . Dequant(W) in FP64 (Eq. 2) ---- */
@@ -135,9 +198,9 @@ void orc_dequant(const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
  * (n0 = 0, n1 = N, k0 = 0, k1 = K for the whole product).  Column n of
  * Dequant(W) is formed once (FP16-rounded, then widened) and every row of A is
  * multiplied into it. */
-void orc_gemm_kslice_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
-                          int M, int N, int K, int group, int k0, int k1, int n0, int n1,
-                          double *C_ref)
+void orc_gemm_kslice_cols_fmt(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                              int M, int N, int K, int group, int k0, int k1, int n0, int n1, int bf16,
+                              double *C_ref)
 {
     #pragma omp parallel
     {
@@ -147,18 +210,32 @@ void orc_gemm_kslice_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t 
             for (int k = k0; k < k1; ++k) {
                 int g = k / group;
                 uint16_t w16 = orc_dequant_one(orc_q_at(Wq, N, k, n),
-                                               Z[(size_t)g * N + n], S[(size_t)g * N + n]);
-                wcol[k] = (double)orc_f16_to_f32(w16);
+                                               Z[(size_t)g * N + n], S[(size_t)g * N + n], bf16);
+                wcol[k] = orc_widen(w16, bf16);
             }
             for (int m = 0; m < M; ++m) {
                 double acc = 0.0;
                 for (int k = k0; k < k1; ++k)
-                    acc += (double)orc_f16_to_f32(A[(size_t)m * K + k]) * wcol[k];
+                    acc += orc_widen(A[(size_t)m * K + k], bf16) * wcol[k];
                 C_ref[(size_t)m * N + n] = acc;
             }
         }
         free(wcol);
     }
+}
+
+void orc_gemm_kslice_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                          int M, int N, int K, int group, int k0, int k1, int n0, int n1,
+                          double *C_ref)
+{
+    orc_gemm_kslice_cols_fmt(A, Wq, S, Z, M, N, K, group, k0, k1, n0, n1, 0, C_ref);
+}
+
+/* The whole product in the chosen 16-bit format (0 = FP16, 1 = BF16). */
+void orc_gemm_fmt(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
+                  int M, int N, int K, int group, int bf16, double *C_ref)
+{
+    orc_gemm_kslice_cols_fmt(A, Wq, S, Z, M, N, K, group, 0, K, 0, N, bf16, C_ref);
 }
 
 void orc_gemm_cols(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, const uint8_t *Z,
@@ -188,8 +265,8 @@ void orc_gemm_kslice(const uint16_t *A, const uint32_t *Wq, const uint16_t *S, c
  * int64 and returns FP16 bits [M, N].  Returns nonzero if Emin..Emax spans more
  * than 30 binary places (would not fit the int64 scaling used here).
  */
-int orc_gemm_int(const int8_t *A, const uint32_t *Wq, const int8_t *E, const uint8_t *Z,
-                 int M, int N, int K, int group, uint16_t *C16)
+int orc_gemm_int_fmt(const int8_t *A, const uint32_t *Wq, const int8_t *E, const uint8_t *Z,
+                     int M, int N, int K, int group, int bf16, uint16_t *C16)
 {
     int G = K / group;
     int emin = 127, emax = -128;
@@ -208,9 +285,15 @@ int orc_gemm_int(const int8_t *A, const uint32_t *Wq, const int8_t *E, const uin
                     part += (int64_t)A[(size_t)m * K + k] * (int64_t)(orc_q_at(Wq, N, k, n) - z);
                 total += part * ((int64_t)1 << (E[(size_t)g * N + n] - emin));
             }
-            C16[(size_t)m * N + n] = orc_f64_to_f16_rn(ldexp((double)total, emin));
+            C16[(size_t)m * N + n] = orc_round16(ldexp((double)total, emin), bf16);
         }
     return 0;
+}
+
+int orc_gemm_int(const int8_t *A, const uint32_t *Wq, const int8_t *E, const uint8_t *Z,
+                 int M, int N, int K, int group, uint16_t *C16)
+{
+    return orc_gemm_int_fmt(A, Wq, E, Z, M, N, K, group, 0, C16);
 }
 
 int orc_num_threads(void)
