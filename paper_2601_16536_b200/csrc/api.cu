@@ -27,7 +27,7 @@ struct DeviceState {
     int max_smem_optin = 0;
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    bool decode_attr_set[3][2][3][2] = {};   // [mb][cluster exchange][log2 SG][bf16]
+    bool decode_attr_set[3][2][3][2][2] = {};   // [mb][cluster exchange][log2 SG][bf16][symmetric]
     bool tile_attr_set[5][3][2] = {};         // [batch-tile index][log2 SG][bf16]
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
     // kernel in its stream has finished.  The previous kernel of a stream may be a w4a16_pack that
@@ -121,6 +121,8 @@ int decode_mb(int M) { return M <= 8 ? 1 : 2; }
 // them.
 struct DecodeGeom {
     int mb, mchunks, stages, smem_bytes, ctas, nchunks;
+    int stage_bytes;   // ring stride for the batch rows a CTA has
+    int prefetch;      // stages whose weights are requested before the wait for the previous kernel
     int cps;       // CTAs per SM the launch is sized for (2 or 3)
     bool cluster;  // one thread-block cluster of split_k CTAs per tile: partial tiles meet in shared memory
     int split_k;   // what the kernel runs: 0 = balanced chunks, S >= 1 = S slices per tile
@@ -188,11 +190,19 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     g.cluster = allow_cluster && split_k >= 2 && split_k <= kDecMaxCluster && g.nchunks == g.ctas && g.mchunks == 1;
     const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
     const int xs = g.cluster ? split_k : 0;   // slices that meet in the exchange buffer
-    int st = (budget - 128 - decode_red_bytes(g.mb) - decode_xch_bytes(g.mb, xs)) / decode_stage_bytes(g.mb, sg);
-    if (st > kDecMaxStages) st = kDecMaxStages;
-    if (st < 2) st = 2;
+    const int rows = M < 8 * g.mb ? M : 8 * g.mb;   // batch rows of a CTA (the last chunk of a large M may have fewer)
+    g.stage_bytes = decode_stage_bytes(rows, sg);
+    int st = kDecMaxStages;
+    while (st > 2 && decode_smem_bytes(g.mb, rows, sg, st, xs) > budget) --st;
     g.stages = st;
-    g.smem_bytes = decode_smem_bytes(g.mb, sg, st, xs);
+    // Weights do not depend on the previous kernel of the stream, so they may be requested before the wait
+    // for it.  With K slices (several CTAs per tile, short chunks) that pays for one stage only: the early
+    // requests take HBM bandwidth from the previous kernel's last CTAs and stand in the copy queue in front
+    // of this kernel's activation rows (K = 11008 / N = 4096, M = 1: one stage 9.15 us, two 9.4, the whole
+    // ring 10.4; K = 16384 / N = 4096: 11.7 / 12.0 / 12.9).  Whole tiles (wide N) gain 2 to 4 % from the
+    // full ring (K = 4096 / N = 22016: 15.45 / 15.2 / 14.9 us).
+    g.prefetch = split_k == 1 ? st : 1;
+    g.smem_bytes = decode_smem_bytes(g.mb, rows, sg, g.stages, xs);
     return g;
 }
 
@@ -547,16 +557,18 @@ namespace {
 
 // ---- kernel tables: one entry per template instantiation ------------------------------------------
 typedef void (*DecodeKernel)(const DecodeParams);
-template <int SG, bool BF>
+template <int SG, bool BF, int SYM>
 DecodeKernel decode_kernel_of(int mb, bool cluster) {
-    return cluster ? (mb == 2 ? gemm_decode_kernel<2, true, SG, BF> : gemm_decode_kernel<1, true, SG, BF>)
-                   : (mb == 2 ? gemm_decode_kernel<2, false, SG, BF> : gemm_decode_kernel<1, false, SG, BF>);
+    return cluster ? (mb == 2 ? gemm_decode_kernel<2, true, SG, BF, SYM> : gemm_decode_kernel<1, true, SG, BF, SYM>)
+                   : (mb == 2 ? gemm_decode_kernel<2, false, SG, BF, SYM> : gemm_decode_kernel<1, false, SG, BF, SYM>);
 }
-DecodeKernel decode_kernel(int mb, bool cluster, int sg, bool bf) {
-    if (bf) return sg == 1 ? decode_kernel_of<1, true>(mb, cluster) : sg == 2 ? decode_kernel_of<2, true>(mb, cluster)
-                                                                              : decode_kernel_of<4, true>(mb, cluster);
-    return sg == 1 ? decode_kernel_of<1, false>(mb, cluster) : sg == 2 ? decode_kernel_of<2, false>(mb, cluster)
-                                                                       : decode_kernel_of<4, false>(mb, cluster);
+// FP16 with groups of 128 has a build for each of the asymmetric and the symmetric format; the other
+// formats share one build that tells the two apart at run time.
+DecodeKernel decode_kernel(int mb, bool cluster, int sg, bool bf, bool sym) {
+    if (bf) return sg == 1 ? decode_kernel_of<1, true, 2>(mb, cluster) : sg == 2 ? decode_kernel_of<2, true, 2>(mb, cluster)
+                                                                                 : decode_kernel_of<4, true, 2>(mb, cluster);
+    if (sg == 1) return sym ? decode_kernel_of<1, false, 1>(mb, cluster) : decode_kernel_of<1, false, 0>(mb, cluster);
+    return sg == 2 ? decode_kernel_of<2, false, 2>(mb, cluster) : decode_kernel_of<4, false, 2>(mb, cluster);
 }
 typedef void (*TileKernel)(const CUtensorMap, const TileParams);
 template <int SG, bool BF>
@@ -699,9 +711,11 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
+    p.stage_bytes = g.stage_bytes;
+    p.prefetch = g.prefetch;
     p.epi = epi;
-    DecodeKernel kern = decode_kernel(g.mb, g.cluster, sg, bf);
-    bool& attr_set = d->decode_attr_set[g.mb][g.cluster ? 1 : 0][log2_sg(sg)][bf ? 1 : 0];
+    DecodeKernel kern = decode_kernel(g.mb, g.cluster, sg, bf, sym);
+    bool& attr_set = d->decode_attr_set[g.mb][g.cluster ? 1 : 0][log2_sg(sg)][bf ? 1 : 0][sym ? 1 : 0];
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
@@ -839,10 +853,12 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     p.split_k = g.split_k;
     p.nchunks = g.nchunks;
     p.stages = g.stages;
+    p.stage_bytes = g.stage_bytes;
+    p.prefetch = g.prefetch;
     p.epi.bias = nullptr;
     p.epi.act = kActNone;
-    DecodeKernel kern = decode_kernel(g.mb, false, sg, false);
-    bool& attr_set = d->decode_attr_set[g.mb][0][log2_sg(sg)][0];
+    DecodeKernel kern = decode_kernel(g.mb, false, sg, false, false);
+    bool& attr_set = d->decode_attr_set[g.mb][0][log2_sg(sg)][0][0];
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {

@@ -61,10 +61,17 @@ struct DecodeParams {
     int split_k;        // 0: balanced chunks; S >= 1: classic Split-K
     int nchunks;        // balanced: gridDim.x; classic: T * split_k
     int stages;
+    int stage_bytes;    // ring stride: decode_stage_bytes(rows of a batch chunk, sg)
+    int prefetch;       // stages whose weights are requested before the wait for the previous kernel
     Epilogue epi;
 };
 
-__host__ __device__ inline int decode_stage_bytes(int mb, int sg) { return dec_stage_a(sg) + 8 * mb * kDecARowBytes; }
+// One ring stage holds the activation rows a CTA really has (min(M, 8 MB)), not 8 MB of them: a call with
+// one batch row gets five stages where eight rows get four.  A multiple of 128 bytes, so that every
+// stage starts on the same shared-memory bank.
+__host__ __device__ inline int decode_stage_bytes(int rows, int sg) {
+    return (dec_stage_a(sg) + rows * kDecARowBytes + 127) / 128 * 128;
+}
 __host__ __device__ inline int decode_red_bytes(int mb) {
     return kDecUnitsPerStage * 8 * mb * kDecRedStride * 4;
 }
@@ -72,9 +79,20 @@ __host__ __device__ inline int decode_red_bytes(int mb) {
 // kDecMaxCluster slices (clusters of 8 are the largest every device places, but measured worse than
 // 6 everywhere: 6.5 against 6.0 us at K = 8192 / N = 2048, 18.8 against 9.2 with two batch blocks)
 constexpr int kDecMaxCluster = 6;
-__host__ __device__ inline int decode_xch_bytes(int mb, int slices) { return slices * 8 * mb * kTileN * 4; }
-__host__ __device__ inline int decode_smem_bytes(int mb, int sg, int stages, int cluster_slices) {
-    return 128 + decode_red_bytes(mb) + decode_xch_bytes(mb, cluster_slices) + stages * decode_stage_bytes(mb, sg);
+// (the first CTA of a cluster keeps its own slice where it is: S - 1 slots)
+__host__ __device__ inline int decode_xch_bytes(int mb, int slices) {
+    return slices > 1 ? (slices - 1) * 8 * mb * kTileN * 4 : 0;
+}
+// Cluster kernels put the reduce buffer on top of the (by then idle) ring: a CTA of a cluster has one
+// slice of one tile, so nothing is in flight when it leaves the tile.  The others leave tiles in
+// mid-stream, with later stages already on their way, and keep a buffer of their own.
+__host__ __device__ inline int decode_smem_bytes(int mb, int rows, int sg, int stages, int cluster_slices) {
+    const int ring = stages * decode_stage_bytes(rows, sg);
+    if (cluster_slices > 1) {
+        const int r = decode_red_bytes(mb);
+        return 128 + decode_xch_bytes(mb, cluster_slices) + (ring > r ? ring : r);
+    }
+    return 128 + decode_red_bytes(mb) + ring;
 }
 
 // D += A . B with A = (a0: row gq, a1: row gq + 8, a2 / a3: the same rows, second k pair).
@@ -204,35 +222,38 @@ struct DecStageIter {
 // then meet in the shared memory of the cluster's first CTA (distributed shared memory + one
 // hardware cluster barrier) instead of going through the workspace, a fence, a ticket and a reload:
 // Phase 3 of Algorithm 1 in about a tenth of the time, still summed in ascending K order.
-// SG = scale / zero-point rows per 128-k block (quantization group 128 / SG); BF = BF16 arithmetic.
-template <int MB, bool CL, int SG, bool BF>
+// SG = scale / zero-point rows per 128-k block (quantization group 128 / SG); BF = BF16 arithmetic;
+// SYM = 0: zero points from the Z buffer, 1: symmetric format (zero point 8, no Z buffer), 2: decided at run
+// time by p.Z == nullptr (one build for both; a few per cent slower than the two dedicated ones).
+template <int MB, bool CL, int SG, bool BF, int SYM>
 __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kRows = 8 * MB;
     constexpr int kStageZ = dec_stage_z(SG), kStageA = dec_stage_a(SG);
-    constexpr int kStageBytes = kStageA + 8 * MB * kDecARowBytes;
-    const bool sym = p.Z == nullptr;
+    const int stage_bytes = p.stage_bytes;
+    const bool sym = SYM == 2 ? (p.Z == nullptr) : (SYM == 1);
     const int mz = blockIdx.y;
     const int m0 = mz * kRows;
     const int rows = min(kRows, p.M - m0);  // batch rows this CTA really has
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = p.stages;
 
-    // shared layout: [barriers + flag, 128 B][reduce buffer][exchange buffer (CL)][stage 0][stage 1]...
+    // shared layout: [barriers + flag, 128 B][reduce buffer | exchange buffer (CL)][stage 0][stage 1]...
+    // (CL: the reduce buffer lies on top of the ring, see decode_smem_bytes)
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);
     uint64_t* empty = full + kDecMaxStages;
-    uint64_t* xbar = full + 2 * kDecMaxStages;   // CL only: the slices' partial tiles have landed (CTA 0's is used)
+    uint64_t* xbar = full + 2 * kDecMaxStages;   // CL only: the other slices' partial tiles have landed (CTA 0's is used)
     int* last_flag = reinterpret_cast<int*>(smem + 120);
-    float* red = reinterpret_cast<float*>(smem + 128);
-    float* xch = reinterpret_cast<float*>(smem + 128 + decode_red_bytes(MB));   // CL only: [slice][8 MB rows][64]
-    unsigned char* stage0 = smem + 128 + decode_red_bytes(MB) + decode_xch_bytes(MB, CL ? p.split_k : 0);
+    float* xch = reinterpret_cast<float*>(smem + 128);   // CL only: [slice 1 .. S - 1][8 MB rows][64]
+    unsigned char* stage0 = smem + 128 + (CL ? decode_xch_bytes(MB, p.split_k) : decode_red_bytes(MB));
+    float* red = reinterpret_cast<float*>(CL ? stage0 : smem + 128);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
             mbar_init(&full[i], 1);
             mbar_init(&empty[i], kDecWarps);
         }
-        if (CL) mbar_init(xbar, (uint32_t)(p.split_k * kDecWarps));   // one arrival per consumer warp of the cluster
+        if (CL) mbar_init(xbar, (uint32_t)((p.split_k - 1) * kDecWarps));   // one arrival per consumer warp of the other CTAs
         fence_mbar_init();
     }
     // (Batch rows this CTA does not have are never loaded: an MMA column only feeds its own output
@@ -269,13 +290,13 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
         // 1. packed weights of the first ring-full of stages: they do not depend on the previous kernel
         {
             DecStageIter pre(p);
-            for (int i = 0; i < stages && pre.valid(); ++i, pre.next()) {
+            for (int i = 0; i < p.prefetch && pre.valid(); ++i, pre.next()) {
                 if (lane == 0) {
                     const int gc = pre.units();
                     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full[i])),
                                  "r"((uint32_t)gc * unit_tx)
                                  : "memory");
-                    issue_weights(pre, stage0 + (size_t)i * kStageBytes, &full[i], gc);
+                    issue_weights(pre, stage0 + (size_t)i * stage_bytes, &full[i], gc);
                 }
             }
         }
@@ -285,11 +306,19 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
         uint32_t phase = 0;
         for (DecStageIter it(p); it.valid(); it.next(), ++n) {
             const int gc = it.units();
-            unsigned char* st = stage0 + (size_t)slot * kStageBytes;
-            if (n < stages) {
+            unsigned char* st = stage0 + (size_t)slot * stage_bytes;
+            if (n < p.prefetch) {
                 if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)(rows * gc * (kGroup * 2)));
                 __syncwarp();
                 issue_rows(it, st, &full[slot], gc);
+            } else if (n < stages) {
+                // first use of this slot, weights not requested yet: nothing to wait for; the (small) row
+                // copies go in front of the weights
+                if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)gc * unit_tx + (uint32_t)(rows * gc * (kGroup * 2)));
+                __syncwarp();
+                issue_rows(it, st, &full[slot], gc);
+                __syncwarp();
+                if (lane == 0) issue_weights(it, st, &full[slot], gc);
             } else {
                 if (!mbar_wait_producer(&empty[slot], phase ^ 1u)) return;  // status recorded
                 if (lane == 0) {
@@ -326,7 +355,10 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
     //   scales / zeros: the lane's four columns 32 hh + gq, + 8, + 16, + 24 are neighbours (sz_perm)
     const uint32_t stage0_addr = smem_u32(stage0);
     const uint32_t w_off = (uint32_t)(us * kBlockBytes + hh * 1024 + (tig >> 1) * 128 + ((gq + 4 * (tig >> 1)) & 7) * 16 + (tig & 1) * 8);
-    const uint32_t a_off = (uint32_t)(kStageA + us * (kGroup * 2) + gq * kDecARowBytes + tig * 32);
+    // (a stage holds only the `rows` batch rows this CTA has: lanes of absent rows read the last present one,
+    // and what they compute lands in output columns that are never stored)
+    const uint32_t a_off = (uint32_t)(kStageA + us * (kGroup * 2) + min(gq, rows - 1) * kDecARowBytes + tig * 32);
+    const uint32_t a_off1 = (uint32_t)(kStageA + us * (kGroup * 2) + min(8 + gq, rows - 1) * kDecARowBytes + tig * 32);
     // SG = 4 (groups of 32 k): the lane's 16 k of a 64-k half lie in row 2 c + tig / 2
     const int jlane = SG == 4 ? (tig >> 1) : 0;
     const uint32_t s_off = (uint32_t)(kDecStageS + (us * SG + jlane) * (kSBlockHalves * 2) + (32 * hh + 4 * gq) * 2);
@@ -393,7 +425,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             const int gc = min(kDecUnitsPerStage, min(u1, tile_end) - u);
             if (!mbar_wait(&full[slot], phase)) return;  // status recorded; every consumer warp sees it
             if (us < gc) {
-                const uint32_t wa = st_addr + w_off, aa = st_addr + a_off;
+                const uint32_t wa = st_addr + w_off, aa = st_addr + a_off, aa1 = st_addr + a_off1;
                 if constexpr (SG == 1) load_consts(st_addr, 0);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
@@ -404,12 +436,13 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
 #pragma unroll
                     for (int mb = 0; mb < MB; ++mb) {
                         uint4 x, y;
+                        const uint32_t ab = mb == 0 ? aa : aa1;
                         if (c == 0) {
-                            x = mb == 0 ? lds128<0>(aa) : lds128<8 * kDecARowBytes>(aa);
-                            y = mb == 0 ? lds128<16>(aa) : lds128<8 * kDecARowBytes + 16>(aa);
+                            x = lds128<0>(ab);
+                            y = lds128<16>(ab);
                         } else {
-                            x = mb == 0 ? lds128<128>(aa) : lds128<8 * kDecARowBytes + 128>(aa);
-                            y = mb == 0 ? lds128<128 + 16>(aa) : lds128<8 * kDecARowBytes + 128 + 16>(aa);
+                            x = lds128<128>(ab);
+                            y = lds128<128 + 16>(ab);
                         }
                         bw[mb][0] = x.x; bw[mb][1] = x.y; bw[mb][2] = x.z; bw[mb][3] = x.w;
                         bw[mb][4] = y.x; bw[mb][5] = y.y; bw[mb][6] = y.z; bw[mb][7] = y.w;
@@ -440,7 +473,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[slot]);
-            st_addr += (uint32_t)kStageBytes;
+            st_addr += (uint32_t)stage_bytes;
             if (++slot == stages) {
                 slot = 0;
                 phase ^= 1u;
@@ -468,29 +501,35 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             // first segment of a chunk -> slot 2 ci, a chunk's continuation into a later tile -> 2 ci + 1
             float* my_slot = ws_mz + (size_t)(2 * ci + (seg_start == u0 ? 0 : 1)) * (kRows * kTileN);
             if (CL && !whole) {
-                // this CTA's slice -> slot `rank` of the exchange buffer of the cluster's CTA 0
-                uint32_t rank, xch0, xbar0;
+                // slices 1 .. S - 1 -> slot rank - 1 of the exchange buffer of the cluster's CTA 0, which
+                // adds them to its own slice 0 in ascending order
+                uint32_t rank;
                 asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xch0) : "r"(smem_u32(xch)), "r"(0u));
-                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xbar0) : "r"(smem_u32(xbar)), "r"(0u));
-                for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
-                    const int n = idx & (kTileN - 1), m = idx >> 6;
-                    float v = red[m * kDecRedStride + n];
+                if (rank != 0) {
+                    uint32_t xch0, xbar0;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xch0) : "r"(smem_u32(xch)), "r"(0u));
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xbar0) : "r"(smem_u32(xbar)), "r"(0u));
+                    for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
+                        const int n = idx & (kTileN - 1), m = idx >> 6;
+                        float v = red[m * kDecRedStride + n];
 #pragma unroll
-                    for (int w = 1; w < kDecUnitsPerStage; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
-                    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(xch0 + (rank * (kRows * kTileN) + idx) * 4u), "f"(v)
-                                 : "memory");
-                }
-                // the warp's stores, then one release-arrival per warp on CTA 0's barrier
-                __syncwarp();
-                if (lane == 0)
-                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(xbar0) : "memory");
-                if (rank == 0) {
+                        for (int w = 1; w < kDecUnitsPerStage; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
+                        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(xch0 + ((rank - 1u) * (kRows * kTileN) + idx) * 4u),
+                                     "f"(v)
+                                     : "memory");
+                    }
+                    // the warp's stores, then one release-arrival per warp on CTA 0's barrier
+                    __syncwarp();
+                    if (lane == 0)
+                        asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(xbar0) : "memory");
+                } else {
                     if (!mbar_wait_cluster(xbar, 0u)) return;   // status recorded
                     for (int idx = threadIdx.x; idx < rows * kTileN; idx += kDecConsumers) {
                         const int n = idx & (kTileN - 1), m = idx >> 6;
-                        float v = xch[idx];
-                        for (int sl = 1; sl < p.split_k; ++sl) v += xch[sl * (kRows * kTileN) + idx];
+                        float v = red[m * kDecRedStride + n];
+#pragma unroll
+                        for (int w = 1; w < kDecUnitsPerStage; ++w) v += red[(w * kRows + m) * kDecRedStride + n];
+                        for (int sl = 1; sl < p.split_k; ++sl) v += xch[(sl - 1) * (kRows * kTileN) + idx];
                         p.C[(size_t)(m0 + m) * p.N + (size_t)t * kTileN + n] = finish<BF>(v, t * kTileN + n, p.epi);
                     }
                 }
