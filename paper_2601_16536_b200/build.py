@@ -36,19 +36,31 @@ def up_to_date() -> bool:
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compile every .cu of csrc/ to an object (in parallel) and link them into the shared library."""
     if not force and up_to_date():
         return LIB
-    tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo",
-           "-gencode", "arch=compute_100a,code=sm_100a",
-           "-shared", "-Xcompiler", "-fPIC",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", tmp] + sources()
+    import concurrent.futures
+    import tempfile
+    flags = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
+             "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
+        flags += ["-Xptxas", "-v"]
+    with tempfile.TemporaryDirectory(prefix="w4a16_build_") as tmpdir:
+        def compile_one(src):
+            obj = os.path.join(tmpdir, os.path.basename(src)[:-3] + ".o")
+            out = subprocess.run([_nvcc()] + flags + ["-c", src, "-o", obj], capture_output=True, text=True)
+            return src, obj, out
+        objs = []
+        with concurrent.futures.ThreadPoolExecutor(max_workers=max(1, min(len(sources()), os.cpu_count() or 1))) as ex:
+            for src, obj, out in ex.map(compile_one, sources()):
+                if verbose or out.returncode != 0:
+                    sys.stderr.write(out.stdout + out.stderr)
+                if out.returncode != 0:
+                    raise RuntimeError("nvcc failed on %s" % src)
+                objs.append(obj)
+        tmp = LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs)
+        os.replace(tmp, LIB)
     return LIB
 
 

@@ -9,8 +9,7 @@
 
 #include "common.cuh"
 #include "kernels_basic.cuh"
-#include "kernel_decode.cuh"
-#include "kernel_tile.cuh"
+#include "kernel_tables.h"
 
 using namespace w4a16;
 
@@ -28,7 +27,7 @@ struct DeviceState {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     bool decode_attr_set[3][2][3][2][2] = {};   // [mb][cluster exchange][log2 SG][bf16][symmetric]
-    bool tile_attr_set[5][3][2] = {};         // [batch-tile index][log2 SG][bf16]
+    bool tile_attr_set[5][3][2][2][2] = {};   // [batch-tile index][log2 SG][bf16][symmetric][epilogue]
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
     // kernel in its stream has finished.  The previous kernel of a stream may be a w4a16_pack that
     // writes those weights, so the first GEMM launched on a stream after any pack on the device is a
@@ -555,33 +554,15 @@ int w4a16_dequant(const void* Wq, const void* S, const void* Z, uint16_t* W16, i
 
 namespace {
 
-// ---- kernel tables: one entry per template instantiation ------------------------------------------
-typedef void (*DecodeKernel)(const DecodeParams);
-template <int SG, bool BF, int SYM>
-DecodeKernel decode_kernel_of(int mb, bool cluster) {
-    return cluster ? (mb == 2 ? gemm_decode_kernel<2, true, SG, BF, SYM> : gemm_decode_kernel<1, true, SG, BF, SYM>)
-                   : (mb == 2 ? gemm_decode_kernel<2, false, SG, BF, SYM> : gemm_decode_kernel<1, false, SG, BF, SYM>);
-}
-// FP16 with groups of 128 has a build for each of the asymmetric and the symmetric format; the other
-// formats share one build that tells the two apart at run time.
+// ---- kernel tables: the instantiations live in the inst_*.cu units --------------------------------
 DecodeKernel decode_kernel(int mb, bool cluster, int sg, bool bf, bool sym) {
-    if (bf) return sg == 1 ? decode_kernel_of<1, true, 2>(mb, cluster) : sg == 2 ? decode_kernel_of<2, true, 2>(mb, cluster)
-                                                                                 : decode_kernel_of<4, true, 2>(mb, cluster);
-    if (sg == 1) return sym ? decode_kernel_of<1, false, 1>(mb, cluster) : decode_kernel_of<1, false, 0>(mb, cluster);
-    return sg == 2 ? decode_kernel_of<2, false, 2>(mb, cluster) : decode_kernel_of<4, false, 2>(mb, cluster);
+    return bf ? decode_kernel_bf16(mb, cluster, sg, sym) : decode_kernel_f16(mb, cluster, sg, sym);
 }
-typedef void (*TileKernel)(const CUtensorMap, const TileParams);
-template <int SG, bool BF>
-TileKernel tile_kernel_of(int mt_index) {
-    return mt_index == 0 ? gemm_tile_kernel<16, SG, BF> : mt_index == 1 ? gemm_tile_kernel<32, SG, BF>
-         : mt_index == 2 ? gemm_tile_kernel<64, SG, BF> : mt_index == 3 ? gemm_tile_kernel<128, SG, BF>
-                                                                         : gemm_tile_kernel<256, SG, BF>;
-}
-TileKernel tile_kernel(int mt_index, int sg, bool bf) {
-    if (bf) return sg == 1 ? tile_kernel_of<1, true>(mt_index) : sg == 2 ? tile_kernel_of<2, true>(mt_index)
-                                                                         : tile_kernel_of<4, true>(mt_index);
-    return sg == 1 ? tile_kernel_of<1, false>(mt_index) : sg == 2 ? tile_kernel_of<2, false>(mt_index)
-                                                                  : tile_kernel_of<4, false>(mt_index);
+TileKernel tile_kernel(int mt_index, int sg, bool bf, bool sym, bool epi) {
+    if (bf) return sg == 1 ? tile_kernel_bf16_sg1(mt_index, sym, epi) : sg == 2 ? tile_kernel_bf16_sg2(mt_index, sym, epi)
+                                                                                : tile_kernel_bf16_sg4(mt_index, sym, epi);
+    return sg == 1 ? tile_kernel_f16_sg1(mt_index, sym, epi) : sg == 2 ? tile_kernel_f16_sg2(mt_index, sym, epi)
+                                                                       : tile_kernel_f16_sg4(mt_index, sym, epi);
 }
 
 // The body of every GEMM entry point; the caller holds g_mu.
@@ -664,8 +645,9 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         p.nchunks = g.nchunks;
         p.stages = g.stages;
         p.epi = epi;
-        TileKernel kern = tile_kernel(g.mt_index, sg, bf);
-        bool& attr_set = d->tile_attr_set[g.mt_index][log2_sg(sg)][bf ? 1 : 0];
+        const bool has_epi = bias != nullptr || act != W4A16_ACT_NONE;
+        TileKernel kern = tile_kernel(g.mt_index, sg, bf, sym, has_epi);
+        bool& attr_set = d->tile_attr_set[g.mt_index][log2_sg(sg)][bf ? 1 : 0][sym ? 1 : 0][has_epi ? 1 : 0];
         if (!attr_set) {
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
                 cudaSuccess) {
@@ -886,12 +868,18 @@ int w4a16_selftest_wait_timeout(unsigned limit_us, w4a16_stream_t stream) {
 int w4a16_device_status(int* status_out) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (!status_out) return W4A16_ERR_NULL;
-    int v = 0, zero = 0;
-    if (cudaDeviceSynchronize() != cudaSuccess ||
-        cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)) != cudaSuccess ||
-        cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) {
+    if (cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
         return W4A16_ERR_CUDA;
+    }
+    // every translation unit that holds kernels has a status word of its own
+    const int words[] = {status_take_this_unit(),     status_take_decode_f16(),   status_take_decode_bf16(),
+                         status_take_tile_f16_sg1(),  status_take_tile_f16_sg2(), status_take_tile_f16_sg4(),
+                         status_take_tile_bf16_sg1(), status_take_tile_bf16_sg2(), status_take_tile_bf16_sg4()};
+    int v = 0;
+    for (int w : words) {
+        if (w < 0) return W4A16_ERR_CUDA;
+        v |= w;
     }
     *status_out = v;
     if (v != 0) {

@@ -56,12 +56,24 @@ __host__ __device__ constexpr int block_word_index(int col, int kw) {
            (kw & 3);
 }
 
-// Status word: a kernel whose bounded wait runs out ORs a code in here and returns.
-__device__ int g_status_word = 0;
+// Status word: a kernel whose bounded wait runs out ORs a code in here and returns.  One word per
+// translation unit of the library (the kernels are compiled in several); w4a16_device_status reads
+// and clears all of them through status_take() of each unit.
+static __device__ int g_status_word = 0;
 constexpr int kStatusMbarTimeout = 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every bounded wait of the GEMM kernels: two seconds
 
 __device__ __forceinline__ void report_status(int code) { atomicOr(&g_status_word, code); }
+// Host: read and clear this translation unit's word (the device must be idle); -1 if a CUDA call fails.
+static inline int status_take_this_unit() {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    return v;
+}
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -29,7 +29,6 @@
 #pragma once
 
 #include "common.cuh"
-#include "kernels_basic.cuh"
 
 namespace w4a16 {
 
@@ -223,15 +222,14 @@ struct DecStageIter {
 // hardware cluster barrier) instead of going through the workspace, a fence, a ticket and a reload:
 // Phase 3 of Algorithm 1 in about a tenth of the time, still summed in ascending K order.
 // SG = scale / zero-point rows per 128-k block (quantization group 128 / SG); BF = BF16 arithmetic;
-// SYM = 0: zero points from the Z buffer, 1: symmetric format (zero point 8, no Z buffer), 2: decided at run
-// time by p.Z == nullptr (one build for both; a few per cent slower than the two dedicated ones).
-template <int MB, bool CL, int SG, bool BF, int SYM>
+// SYM = symmetric format (zero point 8, no Z buffer).
+template <int MB, bool CL, int SG, bool BF, bool SYM>
 __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kRows = 8 * MB;
     constexpr int kStageZ = dec_stage_z(SG), kStageA = dec_stage_a(SG);
     const int stage_bytes = p.stage_bytes;
-    const bool sym = SYM == 2 ? (p.Z == nullptr) : (SYM == 1);
+    constexpr bool sym = SYM;
     const int mz = blockIdx.y;
     const int m0 = mz * kRows;
     const int rows = min(kRows, p.M - m0);  // batch rows this CTA really has

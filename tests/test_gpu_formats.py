@@ -122,3 +122,73 @@ def test_bias_and_activation_are_applied_before_the_final_rounding(path, M, act)
         if act == "relu":
             assert np.all(_f64(C) >= 0)
     del ws
+
+
+# ------------------------------------------------------------------ BF16
+@pytest.mark.parametrize("group,symmetric", [(128, False), (64, False), (32, True)])
+def test_bf16_dequant_is_bit_exact(group, symmetric):
+    K, N = 512, 128
+    d = wl.draw_weights(K, N, seed=900 + group, group=group, symmetric=symmetric, bf16=True)
+    r = np.random.Generator(np.random.PCG64(group + 1))
+    d["S"] = r.integers(0, 0x7F80, size=d["S"].shape, dtype=np.uint64).astype(np.uint16)   # the whole BF16 range
+    pw = _pack(d, N, K, group, symmetric, bf16=True)
+    got = _bits(B.w4a16_dequant(pw))
+    want = oracle.dequant(d["Wq"], d["S"], d["Z"], K, N, group, bf16=True)
+    assert np.array_equal(got, want)
+
+
+# BF16 keeps 8 significant bits: the rounding of C itself is 2^-9 relative, so the tolerances of the FP16
+# product (1e-3 Frobenius, 2e-3 per element) are widened by the ratio of the two formats' precision, 2^3
+BF16_FROB, BF16_ELEM = 8e-3, 1.6e-2
+
+
+def _assert_close_bf16(C, ref, what):
+    frob = np.linalg.norm(C - ref) / max(np.linalg.norm(ref), 1e-30)
+    worst = np.max(np.abs(C - ref) / (1.0 + np.abs(ref)))
+    assert np.all(np.isfinite(C)), what
+    assert frob <= BF16_FROB, "%s: rel Frobenius %.3e" % (what, frob)
+    assert worst <= BF16_ELEM, "%s: worst element %.3e" % (what, worst)
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("group,symmetric", [(128, False), (64, True), (32, False)])
+@pytest.mark.parametrize("M,K,N", [(1, 640, 192), (12, 1152, 128), (40, 768, 256)])
+def test_bf16_gemm_matches_oracle(path, group, symmetric, M, K, N):
+    d = wl.make_problem(M, K, N, seed=M + K + group, group=group, symmetric=symmetric, bf16=True)
+    pw = _pack(d, N, K, group, symmetric, bf16=True)
+    ws = ensure_ws(M, N, K, (0, 1, 3))
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, group, bf16=True)
+    for split_k in (0, 1, 3):
+        C = B.w4a16_gemm(_dev16(d["A"], True), pw, split_k=split_k, path=PATHS[path])
+        torch.cuda.synchronize()
+        assert B.w4a16_device_status() == 0
+        assert C.dtype == torch.bfloat16
+        _assert_close_bf16(_f64(C), ref, "bf16 %s g%d sym%d M%d split %d" % (path, group, symmetric, M, split_k))
+    del ws
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+def test_bf16_exact_inputs_are_bit_equal(path):
+    M, K, N = 6, 1152, 128
+    d = wl.make_exact_problem(M, K, N, seed=77, bf16=True)
+    pw = _pack(d, N, K, 128, False, bf16=True)
+    want = oracle.gemm_int(d["A_int"], d["Wq"], d["E"], d["Z"], M, N, K, 128, bf16=True)
+    ws = ensure_ws(M, N, K, (0, 1, 2, 4, 9))
+    for split_k in (0, 1, 2, 4, 9):
+        C = B.w4a16_gemm(_dev16(d["A"], True), pw, split_k=split_k, path=PATHS[path])
+        torch.cuda.synchronize()
+        assert np.array_equal(_bits(C), want), "split_k=%d" % split_k
+    del ws
+
+
+@pytest.mark.parametrize("M", [4, 16, 128])
+def test_bf16_full_size_layer_whole_output(M):
+    K, N = 4096, 4096
+    d = wl.make_problem(M, K, N, seed=300 + M, bf16=True)
+    pw = _pack(d, N, K, 128, False, bf16=True)
+    ws = ensure_ws(M, N, K, 0)
+    C = B.w4a16_gemm(_dev16(d["A"], True), pw)
+    torch.cuda.synchronize()
+    assert B.w4a16_device_status() == 0
+    _assert_close_bf16(_f64(C), oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128, bf16=True), "bf16 M%d" % M)
+    del ws
