@@ -68,6 +68,8 @@ def lib():
         L.orc_gemm_fmt.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp]
         L.orc_gemm_int_fmt.restype = i
         L.orc_gemm_int_fmt.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp]
+        L.orc_quantize.restype = None
+        L.orc_quantize.argtypes = [vp, i, i, i, i, i, vp, vp, vp]
         L.orc_num_threads.restype = i
         L.orc_num_threads.argtypes = []
         _lib = L
@@ -171,6 +173,17 @@ def gemm_int(A_int, Wq, E, Z, M, N, K, group=128, bf16: bool = False) -> np.ndar
     if rc != 0:
         raise ValueError("exponent range too wide for the exact oracle")
     return C
+
+
+def quantize(W16, K: int, N: int, group: int = 128, symmetric: bool = False, bf16: bool = False):
+    """Eq. 1 per (group, column): 16-bit weights [K, N] -> (Wq uint32 [K/8, N], S uint16 [K/group, N],
+    Z uint8 [K/group, N]) in the raw layout."""
+    W16 = _chk(W16, np.uint16, (K, N))
+    Wq = np.empty((K // 8, N), dtype=np.uint32)
+    S = np.empty((K // group, N), dtype=np.uint16)
+    Z = np.empty((K // group, N), dtype=np.uint8)
+    lib().orc_quantize(_p(W16), K, N, group, 1 if symmetric else 0, 1 if bf16 else 0, _p(Wq), _p(S), _p(Z))
+    return Wq, S, Z
 
 
 def epilogue(C_ref: np.ndarray, bias=None, act: str = "none") -> np.ndarray:

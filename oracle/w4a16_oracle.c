@@ -296,6 +296,63 @@ int orc_gemm_int(const int8_t *A, const uint32_t *Wq, const int8_t *E, const uin
     return orc_gemm_int_fmt(A, Wq, E, Z, M, N, K, group, 0, C16);
 }
 
+/* ---- the step before the path: the affine quantizer of Eq. 1,  x_q = round(x / s) + z ----
+ * The paper gives the formula and says that symmetric quantization fixes z; how s and z are chosen, the
+ * rounding of ties and the clamp are open.  Readings used here, per group of `group` consecutive k of one
+ * column n (the granularity of s and z on the GEMM side):
+ *   asymmetric: s = (max - min) / 15 over the group, rounded to the 16-bit format (this stored value is
+ *               the s of every later step); z = clamp(round(-min / s), 0, 15);
+ *   symmetric:  s = max|x| / 7, z = 8 (codes q - 8 in -8 .. 7);
+ *   a group whose s would be zero (all values equal, or all zero) or not finite gets s = 1;
+ *   q = clamp(round(x / s) + z, 0, 15); round = to nearest, ties to even.
+ * Floating point decides integers here, so the precision is part of the definition: every operation is
+ * a single IEEE binary32 operation (subtract, divide, round-to-integer) in the order written; x and s enter
+ * as the exact values of their 16-bit patterns.
+ */
+static inline float orc_group_scale(float num, float den, int bf16)
+{
+    float s32 = num / den;
+    uint16_t b = orc_round16((double)s32, bf16);
+    float s = (float)orc_widen(b, bf16);
+    if (!(s > 0.0f) || isinf(s)) s = 1.0f;
+    return s;
+}
+
+void orc_quantize(const uint16_t *W16, int K, int N, int group, int symmetric, int bf16,
+                  uint32_t *Wq, uint16_t *S, uint8_t *Z)
+{
+    int G = K / group;
+    memset(Wq, 0, sizeof(uint32_t) * (size_t)(K / 8) * N);
+    for (int g = 0; g < G; ++g)
+        for (int n = 0; n < N; ++n) {
+            float lo = INFINITY, hi = -INFINITY, amax = 0.0f;
+            for (int k = g * group; k < (g + 1) * group; ++k) {
+                float x = (float)orc_widen(W16[(size_t)k * N + n], bf16);
+                if (x < lo) lo = x;
+                if (x > hi) hi = x;
+                if (fabsf(x) > amax) amax = fabsf(x);
+            }
+            float s;
+            int z;
+            if (symmetric) {
+                s = orc_group_scale(amax, 7.0f, bf16);
+                z = 8;
+            } else {
+                s = orc_group_scale(hi - lo, 15.0f, bf16);
+                float zf = nearbyintf(-lo / s);
+                z = zf < 0.0f ? 0 : zf > 15.0f ? 15 : (int)zf;
+            }
+            S[(size_t)g * N + n] = orc_round16((double)s, bf16);   /* s is representable: exact */
+            Z[(size_t)g * N + n] = (uint8_t)z;
+            for (int k = g * group; k < (g + 1) * group; ++k) {
+                float x = (float)orc_widen(W16[(size_t)k * N + n], bf16);
+                float r = nearbyintf(x / s) + (float)z;
+                int q = r < 0.0f ? 0 : r > 15.0f ? 15 : (int)r;
+                Wq[(size_t)(k / 8) * N + n] |= (uint32_t)q << (4 * (k % 8));
+            }
+        }
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP
