@@ -173,6 +173,19 @@ int w4a16_gemm_fmt(const uint16_t *A, const void *Wq, const void *S, const void 
                    const uint16_t *bias, uint16_t *C, int M, int N, int K, int group,
                    int split_k, int path, int flags, int act, w4a16_stream_t stream);
 
+/* The step before the path: the affine quantizer of Eq. 1, x_q = round(x / s) + z, applied per group
+ * of `group` consecutive k and per column to 16-bit weights W16 [K, N] row-major (FP16, or BF16 with
+ * W4A16_FLAG_BF16), writing the RAW layout that w4a16_pack[_fmt] consumes.  The paper gives the formula
+ * only; this library fixes the rest as follows.
+ *   asymmetric  s = (max - min) / 15 over the group, rounded to the 16-bit format;
+ *               z = clamp(round(-min / s), 0, 15)
+ *   symmetric (W4A16_FLAG_SYMMETRIC)  s = max|x| / 7, z = 8; Z_raw is not written and may be NULL
+ *   s == 0 or not finite -> s = 1;  q = clamp(round(x / s) + z, 0, 15);  round = nearest, ties to even;
+ *   every operation is a single IEEE binary32 operation, so the codes are reproducible bit for bit.
+ * Offline (weights are quantized once); not part of the timed path. */
+int w4a16_quantize(const uint16_t *W16, uint32_t *Wq_raw, uint16_t *S_raw, uint8_t *Z_raw,
+                   int N, int K, int group, int flags, w4a16_stream_t stream);
+
 /* End-to-end form of w4a16_gemm for callers whose activations live in HOST memory:
  * copies A_host (FP16 [M, K], ideally pinned) into the caller's device staging buffer
  * A_dev, runs w4a16_gemm into the device staging buffer C_dev, and copies the result

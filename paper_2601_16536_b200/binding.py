@@ -28,7 +28,7 @@ EXPORTS = (
     "w4a16_workspace_bytes", "w4a16_set_workspace", "w4a16_choose_split_k",
     "w4a16_choose_split_k_ex", "w4a16_choose_path", "w4a16_pack", "w4a16_dequant", "w4a16_gemm", "w4a16_gemm_ex",
     "w4a16_gemm_host", "w4a16_gemm_static_ws", "w4a16_device_status", "w4a16_selftest_wait_timeout",
-    "w4a16_pack_fmt", "w4a16_dequant_fmt", "w4a16_gemm_fmt",
+    "w4a16_pack_fmt", "w4a16_dequant_fmt", "w4a16_gemm_fmt", "w4a16_quantize",
 )
 
 _lib = None
@@ -84,6 +84,8 @@ def load():
     L.w4a16_dequant_fmt.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     L.w4a16_gemm_fmt.restype = i
     L.w4a16_gemm_fmt.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp]
+    L.w4a16_quantize.restype = i
+    L.w4a16_quantize.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     L.w4a16_selftest_wait_timeout.restype = i
     L.w4a16_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
     L.w4a16_device_status.restype = i
@@ -191,6 +193,19 @@ def w4a16_pack(Wq_raw: torch.Tensor, S_raw: torch.Tensor, Z_raw: Optional[torch.
         _check(load().w4a16_pack_fmt(_ptr(Wq_raw), _ptr(S_raw), None if sym else _ptr(Z_raw), _ptr(out[0]),
                                      _ptr(out[1]), _ptr(out[2]), N, K, group, flags, _stream()), "w4a16_pack_fmt")
     return PackedWeights(out[0], out[1], out[2], N, K, group, flags)
+
+
+def w4a16_quantize(W16: torch.Tensor, group: int = GROUP, flags: int = 0):
+    """Eq. 1 on 16-bit weights [K, N] (CUDA tensor): returns the raw (Wq int32 [K/8, N], S 16-bit [K/group, N],
+    Z uint8 [K/group, N] or None when symmetric) tensors that ``w4a16_pack`` consumes."""
+    K, N = W16.shape
+    dev = W16.device
+    Wq = torch.empty((K // 8, N), dtype=torch.int32, device=dev)
+    S = torch.empty((K // group, N), dtype=_dtype_of(flags), device=dev)
+    Z = None if flags & FLAG_SYMMETRIC else torch.empty((K // group, N), dtype=torch.uint8, device=dev)
+    _check(load().w4a16_quantize(_ptr(W16), _ptr(Wq), _ptr(S), _ptr(Z), N, K, group, flags, _stream()),
+           "w4a16_quantize")
+    return Wq, S, Z
 
 
 def w4a16_dequant(pw: PackedWeights, out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -195,12 +195,19 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     while (st > 2 && decode_smem_bytes(g.mb, rows, sg, st, xs) > budget) --st;
     g.stages = st;
     // Weights do not depend on the previous kernel of the stream, so they may be requested before the wait
-    // for it.  With K slices (several CTAs per tile, short chunks) that pays for one stage only: the early
-    // requests take HBM bandwidth from the previous kernel's last CTAs and stand in the copy queue in front
-    // of this kernel's activation rows (K = 11008 / N = 4096, M = 1: one stage 9.15 us, two 9.4, the whole
-    // ring 10.4; K = 16384 / N = 4096: 11.7 / 12.0 / 12.9).  Whole tiles (wide N) gain 2 to 4 % from the
-    // full ring (K = 4096 / N = 22016: 15.45 / 15.2 / 14.9 us).
-    g.prefetch = split_k == 1 ? st : 1;
+    // for it.  With K slices that pays only for about as many bytes as HBM delivers during that wait (about
+    // 1 us, 6.5 MB over the whole grid): requests beyond that take bandwidth from the previous kernel's last
+    // CTAs and stand in the copy queue in front of this kernel's activation rows.  Measured, stages requested
+    // early = 1 / 2 / whole ring: K = 11008 / N = 4096 (256 CTAs), M = 1: 9.15 / 9.4 / 10.4 us; K = 16384 /
+    // N = 4096: 11.7 / 12.0 / 12.9; K = 6144 / N = 1536 (144 CTAs), M = 8: 5.7 / 5.25 / 5.25.  Whole tiles
+    // (wide N, split_k = 1) gain 2 to 4 % from the whole ring (K = 4096 / N = 22016: 15.45 / 15.2 / 14.9 us).
+    {
+        const long stage_w = (long)kDecUnitsPerStage * (kBlockBytes + sg * (kSBlockHalves * 2 + kZBlockWords * 4));
+        long pf = 6500000L / ((long)g.ctas * g.mchunks * stage_w);
+        if (pf < 1) pf = 1;
+        if (pf > st || split_k == 1) pf = st;
+        g.prefetch = (int)pf;
+    }
     g.smem_bytes = decode_smem_bytes(g.mb, rows, sg, g.stages, xs);
     return g;
 }
@@ -486,6 +493,28 @@ int w4a16_set_workspace(void* dev_ptr, size_t bytes) {
     d->ws = dev_ptr;
     d->ws_bytes = bytes;
     return W4A16_OK;
+}
+
+int w4a16_quantize(const uint16_t* W16, uint32_t* Wq_raw, uint16_t* S_raw, uint8_t* Z_raw, int N, int K, int group,
+                   int flags, w4a16_stream_t stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!flags_ok(flags)) return W4A16_ERR_SHAPE;
+    const bool sym = (flags & W4A16_FLAG_SYMMETRIC) != 0, bf = (flags & W4A16_FLAG_BF16) != 0;
+    if (!W16 || !Wq_raw || !S_raw || (!sym && !Z_raw)) return W4A16_ERR_NULL;
+    int rc = check_weight_shape(N, K, group);
+    if (rc != W4A16_OK) return rc;
+    if (!aligned16(W16) || !aligned16(Wq_raw) || !aligned16(S_raw) || (!sym && !aligned16(Z_raw))) return W4A16_ERR_ALIGN;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != W4A16_OK) return rc;
+    if (!d->is_sm100) return W4A16_ERR_ARCH;
+    const int G = K / group;
+    const size_t total = (size_t)G * N;
+    const unsigned blocks = (unsigned)((total + 127) / 128);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* z = sym ? nullptr : Z_raw;
+    if (bf) quantize_kernel<true><<<blocks, 128, 0, st>>>(W16, Wq_raw, S_raw, z, N, G, group, sym ? 1 : 0);
+    else quantize_kernel<false><<<blocks, 128, 0, st>>>(W16, Wq_raw, S_raw, z, N, G, group, sym ? 1 : 0);
+    return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 
 int w4a16_pack_fmt(const uint32_t* Wq_raw, const uint16_t* S_raw, const uint8_t* Z_raw, void* Wq, void* S, void* Z,

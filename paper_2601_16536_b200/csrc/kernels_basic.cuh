@@ -78,6 +78,63 @@ __device__ __forceinline__ void load_sz(const uint16_t* __restrict__ S, const ui
     z = Z == nullptr ? (uint32_t)kSymZero : ((Z[row * kZBlockWords + (p >> 3)] >> (4 * (p & 7))) & 15u);
 }
 
+// ------------------------------------------------------------------ quantize (the step before the path)
+// Eq. 1, x_q = round(x / s) + z, per group of `group` consecutive k of one column: one thread per (group,
+// column).  Asymmetric: s = (max - min) / 15 rounded to the 16-bit format, z = clamp(round(-min / s), 0, 15);
+// symmetric: s = max|x| / 7, z = 8; a zero or non-finite s becomes 1; q = clamp(round(x / s) + z, 0, 15),
+// ties to even.  Every operation is one IEEE binary32 operation in this order, because the results are
+// integers decided by floating point.  Output in the raw layout that w4a16_pack consumes.
+template <bool BF>
+__device__ __forceinline__ float group_scale(float num, float den, uint16_t& bits) {
+    bits = cast_out<BF>(__fdiv_rn(num, den));
+    float s = widen<BF>(bits);
+    if (!(s > 0.0f) || isinf(s)) {
+        s = 1.0f;
+        bits = cast_out<BF>(1.0f);
+    }
+    return s;
+}
+
+template <bool BF>
+__global__ void quantize_kernel(const uint16_t* __restrict__ W16, uint32_t* __restrict__ Wq, uint16_t* __restrict__ S,
+                                uint8_t* __restrict__ Z, int N, int G, int group, int symmetric) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // (g, n), n fastest
+    if (idx >= (size_t)G * N) return;
+    const int n = (int)(idx % (size_t)N), g = (int)(idx / (size_t)N);
+    const uint16_t* col = W16 + (size_t)g * group * N + n;
+    float lo = INFINITY, hi = -INFINITY, amax = 0.0f;
+    for (int k = 0; k < group; ++k) {
+        const float x = widen<BF>(col[(size_t)k * N]);
+        lo = x < lo ? x : lo;
+        hi = x > hi ? x : hi;
+        amax = fabsf(x) > amax ? fabsf(x) : amax;
+    }
+    uint16_t sb;
+    float s;
+    int z;
+    if (symmetric) {
+        s = group_scale<BF>(amax, 7.0f, sb);
+        z = kSymZero;
+    } else {
+        s = group_scale<BF>(__fsub_rn(hi, lo), 15.0f, sb);
+        const float zf = rintf(__fdiv_rn(-lo, s));
+        z = zf < 0.0f ? 0 : zf > 15.0f ? 15 : (int)zf;
+    }
+    S[idx] = sb;
+    if (Z != nullptr) Z[idx] = (uint8_t)z;
+    for (int kw = 0; kw < group / 8; ++kw) {
+        uint32_t w = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float x = widen<BF>(col[(size_t)(kw * 8 + i) * N]);
+            const float r = __fadd_rn(rintf(__fdiv_rn(x, s)), (float)z);
+            const int q = r < 0.0f ? 0 : r > 15.0f ? 15 : (int)r;
+            w |= (uint32_t)q << (4 * i);
+        }
+        Wq[((size_t)g * (group / 8) + kw) * N + n] = w;
+    }
+}
+
 // ------------------------------------------------------------------ dequant
 // Algorithm 1, Phase 1 as a standalone kernel: one thread per packed word, eight results
 // w16 = rn((q - z) * s) in the 16-bit format: (q - z) is formed exactly and multiplied by s with one
