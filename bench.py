@@ -39,13 +39,11 @@ WORKLOAD = "config2_down_proj_decode_K11008_N4096_M1-2-4-8-16"
 MIN_ROTATION_BYTES = 512 << 20
 PATH_NAMES = {1: "gemm_simple_kernel", 2: "gemm_decode_kernel", 3: "gemm_tile_kernel"}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until captured)
-# DRAM read + write of one M=16 K=11008 N=4096 launch, by the kernel the library picks for it (ncu; None = not
-# captured since that kernel last changed)
-NCU_TRAFFIC_BYTES = {"gemm_tile_kernel": 24134016,      # read 24.13 MB, write 0
-                     "gemm_decode_kernel": 23817984}    # read 23.82 MB, write 0 (<2, 2, cluster>)
-NCU_TRAFFIC_BYTES_TILE = 192325632    # gemm_tile_kernel<256>, M=4096 K=N=8192 (read 136.1 MB + write 56.2 MB)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
+# (None = not captured since that kernel last changed).  Decode kernel: the mean of the five launches of a
+# step, M = 1 / 2 / 4 / 8 / 16 at K = 11008, N = 4096: 23.489 / 23.512 / 23.556 / 23.643 / 23.820 MB read, 0 written.
+NCU_TRAFFIC_BYTES = {"gemm_decode_kernel": 23604000}
+NCU_TRAFFIC_BYTES_TILE = 191389000    # gemm_tile_kernel<256>, M=4096 K=N=8192 (read 132.5 MB + write 58.9 MB)
 
 
 def _peaks():
@@ -402,6 +400,34 @@ def run_ours(args):
                                      5, max(64, args.case_calls // 4), torch)
                 cases[i]["us_warm_l2"] = _r(sec * 1e6, 3)
 
+            # format variants on the same shape (Eq. 1's symmetric case, smaller groups, BF16): same value recipe,
+            # their own algorithmic bytes (no Z traffic when symmetric, more scales with smaller groups)
+            for vname, group, sym, bf in (("symmetric_g128", 128, True, False), ("asymmetric_g64", 64, False, False),
+                                          ("asymmetric_g32", 32, False, False), ("bf16_g128", 128, False, True)):
+                flags = (B.FLAG_SYMMETRIC if sym else 0) | (B.FLAG_BF16 if bf else 0)
+                raw = wl.draw_weights(K, N, 2100, group, sym, bf)
+                dt = torch.bfloat16 if bf else torch.float16
+                rw = _to_dev(raw["Wq"], torch)
+                rs = torch.from_numpy(raw["S"].view(np.int16)).cuda().view(dt)
+                rz = None if sym else _to_dev(raw["Z"], torch)
+                per = wl.algorithmic_bytes(0, K, N, group, sym)
+                packs = [B.w4a16_pack(rw, rs, rz, N, K, group, flags) for _ in range(max(2, -(-MIN_ROTATION_BYTES // per)))]
+                turn = [0]
+
+                def take_v():
+                    turn[0] += 1
+                    return packs[turn[0] % len(packs)]
+                for M in (1, 8, 16):
+                    Av = torch.from_numpy(wl.draw_activations(M, K, 2100 + M, bf16=bf).view(np.int16)).cuda().view(dt)
+                    Cv = torch.empty((M, N), dtype=dt, device="cuda")
+                    med, mn = _time_calls(lambda: B.w4a16_gemm(Av, take_v(), Cv), 10, max(64, args.case_calls // 4), torch)
+                    byts = wl.algorithmic_bytes(M, K, N, group, sym)
+                    cases.append({"config": "2-variant", "layer": vname, "M": M, "K": K, "N": N, "us": _r(med * 1e6, 3),
+                                  "us_min": _r(mn * 1e6, 3), "algorithmic_bytes": byts, "eff_GBps": _r(byts / med / 1e9, 1),
+                                  "roofline_frac": _r(byts / (hbm_peak * 1e9) / med), "bound": "hbm"})
+                del packs, rw, rs, rz
+                torch.cuda.empty_cache()
+
             # cuBLAS / PyTorch FP16 x FP16 on pre-dequantized weights: a reference point, not our path
             if not args.no_cublas:
                 w16 = [B.w4a16_dequant(layer.packed[0]).clone() for _ in range(6)]
@@ -488,8 +514,7 @@ def run_ours(args):
     achieved = bytes_per_launch / launch_us / 1e3
     heavy = SWEEP_M[-1]
     roofline = {"bound": "hbm", "kernel": dom_kernel,
-                "launches": "the %d launches of a step (M = %s), averaged over the timed region"
-                            % (launches_per_step, "/".join(str(m) for m in SWEEP_M)),
+                "launches": "the %d launches of a step, averaged over the timed region" % launches_per_step,
                 "achieved": _r(achieved, 1), "peak": hbm_peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                 "frac": _r(achieved / hbm_peak), "frac_of_nominal_8TBps": _r(achieved / 8000.0),
                 "traffic": NCU_TRAFFIC_BYTES.get(dom_kernel),
