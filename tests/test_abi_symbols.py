@@ -64,6 +64,41 @@ def test_choose_split_k_is_always_acceptable(lib):
     assert lib.w4a16_workspace_bytes(4, 4096, 4096, 128, 4) >= 4 * 4 * 4096 * 4
 
 
+def test_schedule_queries_are_consistent_on_a_grid_of_shapes(lib):
+    """Host logic over 675 (M, N, K, group) combinations, none of them tuned for: the path is one of the two
+    GEMM kernels, the reported split is one w4a16_gemm accepts (1 .. K/128 for every group size), a split of
+    1 needs no workspace, any other split needs at least the ticket header, and the size is bounded by the
+    partial tiles the schedule can produce (two per CTA slot of a 148-SM device, per batch chunk)."""
+    header = 16384 + 131072
+    n = 0
+    for group in (32, 64, 128):
+        for M in (1, 3, 8, 9, 16, 17, 64, 300, 4096):
+            for N in (64, 1536, 4096, 4608, 22016):
+                for K in (128, 1024, 4096, 11008, 28672):
+                    n += 1
+                    blocks = K // 128
+                    assert lib.w4a16_choose_path(M, N, K, group) in (2, 3)
+                    s = lib.w4a16_choose_split_k(M, N, K, group)
+                    assert 1 <= s <= blocks, (M, N, K, group, s)
+                    for path in (1, 2, 3):
+                        assert 1 <= lib.w4a16_choose_split_k_ex(M, N, K, group, path) <= blocks
+                    assert lib.w4a16_workspace_bytes(M, N, K, group, 1) == 0
+                    assert lib.w4a16_workspace_bytes(M, N, K, group, blocks + 1) == 0      # not a valid split
+                    for split in {0, s, min(2, blocks), blocks}:
+                        if split == 1:
+                            continue
+                        need = lib.w4a16_workspace_bytes(M, N, K, group, split)
+                        assert need == 0 or need >= header
+                        # plain path: split x M x N floats; warp-MMA path: two 16 x 64 tiles per chunk and batch
+                        # chunk; tcgen05 path: two MT x 128 tiles per chunk
+                        sp = split if split else max(s, 1)
+                        bound = header + 256 + max(4 * sp * M * N,
+                                                   2 * max(296, (N // 64) * sp) * ((M + 15) // 16) * 16 * 64 * 4,
+                                                   2 * max(148, ((M + 15) // 16) * ((N + 127) // 128) * sp) * 256 * 128 * 4)
+                        assert need <= bound, (M, N, K, group, split, need, bound)
+    assert n == 675
+
+
 def test_path_and_schedule_rules_at_the_benchmark_shapes(lib):
     """Host logic only (148 SMs assumed without a device, which is also what a B200 reports): the
     path and the split the library reports for a shape are the ones it runs (w4a16_gemm asks the same
