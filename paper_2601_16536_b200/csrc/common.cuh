@@ -97,22 +97,13 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait: returns false (after recording the status code) if the phase does not complete
-// within about two seconds.  Fast path: one try_wait (about 40 clocks when the phase is already
-// complete).  Slow path: try_wait with a suspend-time hint, so that a waiting warp sleeps in the
-// barrier unit instead of spending issue slots on polling, and a wall-clock limit read from
+// within about two seconds.  Fast path, inlined: one try_wait (about 40 clocks when the phase is
+// already complete).  Slow path, a function of its own so that the many waits of a kernel do not
+// each carry a copy of the loop: try_wait with a suspend-time hint, so that a waiting warp sleeps in
+// the barrier unit instead of spending issue slots on polling, and a wall-clock limit read from
 // %globaltimer (the hint is only a hint: an iteration count would not bound the time).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, unsigned long long limit_ns) {
     uint32_t ok;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t"
-        "}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    if (ok) return true;
     unsigned long long t0;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
     for (;;) {
@@ -123,7 +114,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
             "selp.u32 %0, 1, 0, p;\n\t"
             "}"
             : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
+            : "r"(bar_addr), "r"(parity), "r"(20000u)
             : "memory");
         if (ok) return true;
         unsigned long long t1;
@@ -132,6 +123,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
     }
     report_status(kStatusMbarTimeout);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs) {
+    uint32_t ok;
+    const uint32_t addr = smem_u32(bar);
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    return mbar_wait_slow(addr, parity, limit_ns);
 }
 
 // The same bounded wait with cluster-scope acquire: for a barrier that CTAs of the cluster arrive on

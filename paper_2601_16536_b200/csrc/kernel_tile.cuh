@@ -208,20 +208,58 @@ __host__ __device__ constexpr uint32_t tile_idesc(int mt, bool bf) {
 }
 
 // ------------------------------------------------------------------ chunk schedule
-// First unit of chunk i (i == nchunks gives the end of the last chunk).
+// (The out-of-line functions below take the schedule in scalars: registers, not a reference to the kernel's
+// parameter block, which would be copied to local memory for every call.)
+// First unit of chunk i (i == nchunks gives the end of the last chunk).  (64-bit divisions: these two and
+// tile_chunk_start below are functions of their own, called once per chunk -- inlined into every role's
+// walk they made up three quarters of the kernel's code, more than the instruction cache holds.)
+static __device__ __noinline__ long long tile_chunk_begin_s(int split_k, int G, int nchunks, long long units, int i) {
+    if (split_k == 0) return ((long long)i * units) / nchunks;
+    const int t = i / split_k, s = i - t * split_k;
+    const int base = G / split_k, rem = G % split_k;
+    return (long long)t * G + s * base + min(s, rem);
+}
 __device__ __forceinline__ long long tile_chunk_begin(const TileParams& p, int i) {
-    if (p.split_k == 0) return ((long long)i * ((long long)p.m_tiles * p.n_tiles * p.G)) / p.nchunks;
-    const int t = i / p.split_k, s = i - t * p.split_k;
-    const int base = p.G / p.split_k, rem = p.G % p.split_k;
-    return (long long)t * p.G + s * base + min(s, rem);
+    return tile_chunk_begin_s(p.split_k, p.G, p.nchunks, (long long)p.m_tiles * p.n_tiles * p.G, i);
 }
 // The chunk that holds unit u.
-__device__ __forceinline__ int tile_chunk_of(const TileParams& p, long long u) {
-    if (p.split_k == 0) return (int)(((u + 1) * p.nchunks - 1) / ((long long)p.m_tiles * p.n_tiles * p.G));
-    const int t = (int)(u / p.G), g = (int)(u - (long long)t * p.G);
-    const int base = p.G / p.split_k, rem = p.G % p.split_k;
+static __device__ __noinline__ int tile_chunk_of_s(int split_k, int G, int nchunks, long long units, long long u) {
+    if (split_k == 0) return (int)(((u + 1) * nchunks - 1) / units);
+    const int t = (int)(u / G), g = (int)(u - (long long)t * G);
+    const int base = G / split_k, rem = G % split_k;
     const int s = (g < rem * (base + 1)) ? g / (base + 1) : rem + (g - rem * (base + 1)) / max(base, 1);
-    return t * p.split_k + s;
+    return t * split_k + s;
+}
+__device__ __forceinline__ int tile_chunk_of(const TileParams& p, long long u) {
+    return tile_chunk_of_s(p.split_k, p.G, p.nchunks, (long long)p.m_tiles * p.n_tiles * p.G, u);
+}
+
+// Where chunk ci (or the next non-empty one of this CTA, stepping by `stride`) starts.
+struct ChunkStart {
+    int ci;        // the chunk found (>= nchunks: none left)
+    int t;         // tile = batch tile * NT + column tile
+    int nt, mt_i;  // t % NT, t / NT
+    int g0;        // first group inside the tile
+    int len;       // units of the chunk
+};
+static __device__ __noinline__ ChunkStart tile_chunk_start(int split_k, int G, int nchunks, int n_tiles, long long units,
+                                                           int ci, int stride) {
+    ChunkStart c;
+    long long u0 = 0;
+    int len = 0;
+    while (ci < nchunks) {
+        u0 = tile_chunk_begin_s(split_k, G, nchunks, units, ci);
+        len = (int)(tile_chunk_begin_s(split_k, G, nchunks, units, ci + 1) - u0);
+        if (len > 0) break;
+        ci += stride;
+    }
+    c.ci = ci;
+    c.len = len;
+    c.t = (int)(u0 / G);
+    c.g0 = (int)(u0 - (long long)c.t * G);
+    c.mt_i = c.t / n_tiles;
+    c.nt = c.t - c.mt_i * n_tiles;
+    return c;
 }
 
 // Walks the segments of this CTA's chunks in order (a segment = the part of a chunk inside one
@@ -245,21 +283,16 @@ struct SegWalk {
         load_chunk();
     }
     __device__ __forceinline__ void load_chunk() {
-        long long u0 = 0;
-        int len = 0;
-        while (ci < p.nchunks) {
-            u0 = tile_chunk_begin(p, ci);
-            len = (int)(tile_chunk_begin(p, ci + 1) - u0);
-            if (len > 0) break;
-            ci += (int)gridDim.x;
-        }
+        const ChunkStart c = tile_chunk_start(p.split_k, p.G, p.nchunks, p.n_tiles, (long long)p.m_tiles * p.n_tiles * p.G, ci,
+                                              (int)gridDim.x);
+        ci = c.ci;
         if (ci >= p.nchunks) return;
-        t = (int)(u0 / p.G);
-        g0 = (int)(u0 - (long long)t * p.G);
-        mt_i = t / p.n_tiles;
-        nt = t - mt_i * p.n_tiles;
-        units = min(len, p.G - g0);
-        left = len - units;
+        t = c.t;
+        g0 = c.g0;
+        mt_i = c.mt_i;
+        nt = c.nt;
+        units = min(c.len, p.G - g0);
+        left = c.len - units;
         first = true;
     }
     __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
