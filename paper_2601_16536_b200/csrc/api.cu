@@ -5,6 +5,8 @@
 
 #include <cuda_runtime.h>
 
+#include <string.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -26,7 +28,7 @@ struct DeviceState {
     int max_smem_optin = 0;
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    bool decode_attr_set[3][2][3][2][2] = {};   // [mb][cluster exchange][log2 SG][bf16][symmetric]
+    bool decode_attr_set[3][2][3][2][2][2] = {};   // [mb][cluster exchange][log2 SG][bf16][symmetric][tensor-copy rows]
     bool tile_attr_set[5][3][2][2][2] = {};   // [batch-tile index][log2 SG][bf16][symmetric][epilogue]
     // Programmatic dependent launch lets a GEMM kernel prefetch packed weights before the previous
     // kernel in its stream has finished.  The previous kernel of a stream may be a w4a16_pack that
@@ -122,10 +124,18 @@ struct DecodeGeom {
     int mb, mchunks, stages, smem_bytes, ctas, nchunks;
     int stage_bytes;   // ring stride for the batch rows a CTA has
     int prefetch;      // stages whose weights are requested before the wait for the previous kernel
+    bool a_box;        // activation rows of a stage as one tensor copy (kernel_decode.cuh)
     int cps;       // CTAs per SM the launch is sized for (2 or 3)
     bool cluster;  // one thread-block cluster of split_k CTAs per tile: partial tiles meet in shared memory
     int split_k;   // what the kernel runs: 0 = balanced chunks, S >= 1 = S slices per tile
 };
+
+// From how many batch rows per CTA on a stage's activation rows come as one tensor copy instead of one bulk
+// copy per row.  Measured (us, bulk copies per row / one tensor copy), K = 11008 / N = 4096: M = 2 9.28 / 9.09,
+// M = 4 9.60 / 9.09, M = 8 10.5 / 9.34, M = 16 13.0 / 11.1; K = 4096 / N = 4096, M = 3: 5.57 / 5.38.  With one
+// row the two are within 1 % (9.15 / 9.09 there, 32.6 / 32.8 at K = 28672 / N = 8192, 14.9 / 15.2 at K = 4096 /
+// N = 22016: the box takes 8 KiB of a slot whatever M is, and long shapes want the ring stage that costs).
+constexpr int kDecABoxMinRows = 2;
 
 DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_cluster = true, int sg = 1) {
     DecodeGeom g;
@@ -190,9 +200,11 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
     const int budget = (227 * 1024) / g.cps - 1024;   // per CTA
     const int xs = g.cluster ? split_k : 0;   // slices that meet in the exchange buffer
     const int rows = M < 8 * g.mb ? M : 8 * g.mb;   // batch rows of a CTA (the last chunk of a large M may have fewer)
-    g.stage_bytes = decode_stage_bytes(rows, sg);
+    // (the box is 8 chunks of 64 k long: K >= 512)
+    g.a_box = rows >= kDecABoxMinRows && G >= kDecUnitsPerStage;
+    g.stage_bytes = decode_stage_bytes(rows, sg, g.a_box);
     int st = kDecMaxStages;
-    while (st > 2 && decode_smem_bytes(g.mb, rows, sg, st, xs) > budget) --st;
+    while (st > 2 && decode_smem_bytes(g.mb, rows, sg, st, xs, g.a_box) > budget) --st;
     g.stages = st;
     // Weights do not depend on the previous kernel of the stream, so they may be requested before the wait
     // for it.  With K slices that pays only for about as many bytes as HBM delivers during that wait (about
@@ -208,7 +220,7 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
         if (pf > st || split_k == 1) pf = st;
         g.prefetch = (int)pf;
     }
-    g.smem_bytes = decode_smem_bytes(g.mb, rows, sg, g.stages, xs);
+    g.smem_bytes = decode_smem_bytes(g.mb, rows, sg, g.stages, xs, g.a_box);
     return g;
 }
 
@@ -365,6 +377,20 @@ bool make_act_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mt) 
     const cuuint64_t dims[3] = {(cuuint64_t)kTileBoxK, (cuuint64_t)M, (cuuint64_t)(K / kTileBoxK)};
     const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)kTileBoxK * 2};
     const cuuint32_t box[3] = {(cuuint32_t)kTileBoxK, (cuuint32_t)mt, (cuuint32_t)(tile_stage_k(mt) / kTileBoxK)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(A), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same activations for the warp-MMA kernel's tensor copy: [K / 64][M][64], box = the 8 chunks of a
+// stage x 8 mb rows x 64 k.
+bool make_decode_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mb) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)M, (cuuint64_t)(K / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)(8 * mb), (cuuint32_t)kDecABoxChunks};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(A), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -584,8 +610,8 @@ int w4a16_dequant(const void* Wq, const void* S, const void* Z, uint16_t* W16, i
 namespace {
 
 // ---- kernel tables: the instantiations live in the inst_*.cu units --------------------------------
-DecodeKernel decode_kernel(int mb, bool cluster, int sg, bool bf, bool sym) {
-    return bf ? decode_kernel_bf16(mb, cluster, sg, sym) : decode_kernel_f16(mb, cluster, sg, sym);
+DecodeKernel decode_kernel(int mb, bool cluster, int sg, bool bf, bool sym, bool a_box) {
+    return bf ? decode_kernel_bf16(mb, cluster, sg, sym, a_box) : decode_kernel_f16(mb, cluster, sg, sym, a_box);
 }
 TileKernel tile_kernel(int mt_index, int sg, bool bf, bool sym, bool epi) {
     if (bf) return sg == 1 ? tile_kernel_bf16_sg1(mt_index, sym, epi) : sg == 2 ? tile_kernel_bf16_sg2(mt_index, sym, epi)
@@ -725,8 +751,14 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     p.stage_bytes = g.stage_bytes;
     p.prefetch = g.prefetch;
     p.epi = epi;
-    DecodeKernel kern = decode_kernel(g.mb, g.cluster, sg, bf, sym);
-    bool& attr_set = d->decode_attr_set[g.mb][g.cluster ? 1 : 0][log2_sg(sg)][bf ? 1 : 0][sym ? 1 : 0];
+    CUtensorMap tmap_a;
+    if (g.a_box) {
+        if (!make_decode_tensor_map(&tmap_a, A, M, K, g.mb)) return W4A16_ERR_CUDA;
+    } else {
+        memset(&tmap_a, 0, sizeof(tmap_a));
+    }
+    DecodeKernel kern = decode_kernel(g.mb, g.cluster, sg, bf, sym, g.a_box);
+    bool& attr_set = d->decode_attr_set[g.mb][g.cluster ? 1 : 0][log2_sg(sg)][bf ? 1 : 0][sym ? 1 : 0][g.a_box ? 1 : 0];
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
@@ -758,7 +790,7 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmap_a, p) != cudaSuccess) {
         cudaGetLastError();
         if (g.cluster) {
             // the device would not place the clusters: from now on the workspace exchange (and the path
@@ -866,10 +898,16 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     p.stages = g.stages;
     p.stage_bytes = g.stage_bytes;
     p.prefetch = g.prefetch;
+    CUtensorMap tmap_a;
+    if (g.a_box) {
+        if (!make_decode_tensor_map(&tmap_a, A, M, K, g.mb)) return W4A16_ERR_CUDA;
+    } else {
+        memset(&tmap_a, 0, sizeof(tmap_a));
+    }
     p.epi.bias = nullptr;
     p.epi.act = kActNone;
-    DecodeKernel kern = decode_kernel(g.mb, false, sg, false, false);
-    bool& attr_set = d->decode_attr_set[g.mb][0][log2_sg(sg)][0][0];
+    DecodeKernel kern = decode_kernel(g.mb, false, sg, false, false, g.a_box);
+    bool& attr_set = d->decode_attr_set[g.mb][0][log2_sg(sg)][0][0][g.a_box ? 1 : 0];
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, d->max_smem_optin) !=
             cudaSuccess) {
@@ -878,7 +916,7 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
         }
         attr_set = true;
     }
-    kern<<<dim3(g.ctas, g.mchunks, 1), kDecThreads, g.smem_bytes, st>>>(p);
+    kern<<<dim3(g.ctas, g.mchunks, 1), kDecThreads, g.smem_bytes, st>>>(tmap_a, p);
     return cudaGetLastError() == cudaSuccess ? W4A16_OK : W4A16_ERR_CUDA;
 }
 

@@ -8,8 +8,9 @@
 //   - classic Split-K (split_k = S): every tile's K range is cut into S slices of whole
 //     groups (Algorithm 1, Phase 2), T*S chunks dealt round-robin to the CTAs.
 // A producer warp brings 4 units per stage (16 KiB of nibbles + their scales and zeros,
-// three TMA bulk copies) plus the matching activation rows into a shared-memory ring
-// guarded by mbarriers; stages never straddle a tile.  Eight consumer warps work on a
+// three TMA bulk copies) plus the matching activation rows (one bulk copy per row, or one
+// tensor copy for all of them: ABOX below) into a shared-memory ring guarded by mbarriers;
+// stages never straddle a tile.  Eight consumer warps work on a
 // stage, two per unit, each on two of the block's four 16-column sub-tiles: two 64-bit shared
 // loads give a lane the nibbles of columns gq and gq + 8 at its 16 k, a logic op and two FP16
 // ops per register turn them into w16 = fp16_rn((q - z) s), and an m16n8k16 tensor-core MMA
@@ -65,11 +66,19 @@ struct DecodeParams {
     Epilogue epi;
 };
 
+// Activation rows of a stage, two ways (template parameter ABOX of the kernel).  Few rows: one bulk copy per row into the tail of the weight stage
+// (1 KiB + 16 B apart).  More rows: every bulk copy costs the producer warp about 50 clocks whatever its
+// size, and 19 of them per 16 KiB stage leave the first ring-full a microsecond late; so the rows then come
+// as ONE tensor copy (A seen as [K / 64][M][64], box = 8 chunks x 8 MB rows x 64 k, 128-byte swizzle, rows
+// past M read as zero) into a second ring of 8 MB KiB slots, 1024-byte aligned, behind the weight ring.
+constexpr int kDecABoxChunks = 2 * kDecUnitsPerStage;    // 64-k chunks per stage
+__host__ __device__ constexpr int dec_a_box_bytes(int mb) { return kDecABoxChunks * 8 * mb * 128; }
+
 // One ring stage holds the activation rows a CTA really has (min(M, 8 MB)), not 8 MB of them: a call with
 // one batch row gets five stages where eight rows get four.  A multiple of 128 bytes, so that every
 // stage starts on the same shared-memory bank.
-__host__ __device__ inline int decode_stage_bytes(int rows, int sg) {
-    return (dec_stage_a(sg) + rows * kDecARowBytes + 127) / 128 * 128;
+__host__ __device__ inline int decode_stage_bytes(int rows, int sg, bool a_box = false) {
+    return (dec_stage_a(sg) + (a_box ? 0 : rows * kDecARowBytes) + 127) / 128 * 128;
 }
 __host__ __device__ inline int decode_red_bytes(int mb) {
     return kDecUnitsPerStage * 8 * mb * kDecRedStride * 4;
@@ -85,8 +94,10 @@ __host__ __device__ inline int decode_xch_bytes(int mb, int slices) {
 // Cluster kernels put the reduce buffer on top of the (by then idle) ring: a CTA of a cluster has one
 // slice of one tile, so nothing is in flight when it leaves the tile.  The others leave tiles in
 // mid-stream, with later stages already on their way, and keep a buffer of their own.
-__host__ __device__ inline int decode_smem_bytes(int mb, int rows, int sg, int stages, int cluster_slices) {
-    const int ring = stages * decode_stage_bytes(rows, sg);
+__host__ __device__ inline int decode_smem_bytes(int mb, int rows, int sg, int stages, int cluster_slices,
+                                                 bool a_box = false) {
+    // (a_box: the second ring and up to 1023 bytes in front of it for its alignment)
+    const int ring = stages * decode_stage_bytes(rows, sg, a_box) + (a_box ? stages * dec_a_box_bytes(mb) + 1024 : 0);
     if (cluster_slices > 1) {
         const int r = decode_red_bytes(mb);
         return 128 + decode_xch_bytes(mb, cluster_slices) + (ring > r ? ring : r);
@@ -222,9 +233,10 @@ struct DecStageIter {
 // hardware cluster barrier) instead of going through the workspace, a fence, a ticket and a reload:
 // Phase 3 of Algorithm 1 in about a tenth of the time, still summed in ascending K order.
 // SG = scale / zero-point rows per 128-k block (quantization group 128 / SG); BF = BF16 arithmetic;
-// SYM = symmetric format (zero point 8, no Z buffer).
-template <int MB, bool CL, int SG, bool BF, bool SYM>
-__global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const DecodeParams p) {
+// SYM = symmetric format (zero point 8, no Z buffer); ABOX = activation rows by tensor copy.
+template <int MB, bool CL, int SG, bool BF, bool SYM, bool ABOX>
+__global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                                                                     const DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kRows = 8 * MB;
     constexpr int kStageZ = dec_stage_z(SG), kStageA = dec_stage_a(SG);
@@ -245,6 +257,12 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
     float* xch = reinterpret_cast<float*>(smem + 128);   // CL only: [slice 1 .. S - 1][8 MB rows][64]
     unsigned char* stage0 = smem + 128 + (CL ? decode_xch_bytes(MB, p.split_k) : decode_red_bytes(MB));
     float* red = reinterpret_cast<float*>(CL ? stage0 : smem + 128);
+    constexpr bool a_box = ABOX;
+    constexpr uint32_t kABoxBytes = (uint32_t)dec_a_box_bytes(MB);
+    // where the activation rows of slot 0 start, and the step to the next slot
+    const uint32_t a_slot0 = a_box ? ((smem_u32(stage0) + (uint32_t)(stages * stage_bytes) + 1023u) & ~1023u)
+                                   : smem_u32(stage0) + (uint32_t)kStageA;
+    const uint32_t a_step = a_box ? kABoxBytes : (uint32_t)stage_bytes;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
@@ -278,13 +296,24 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             if (!sym)
                 bulk_g2s(st + kStageZ, p.Z + (size_t)it.u * (SG * kZBlockWords), (uint32_t)(gc * SG * kZBlockWords * 4), bar);
         };
-        auto issue_rows = [&](const DecStageIter& it, unsigned char* st, uint64_t* bar, int gc) {
+        auto issue_rows = [&](const DecStageIter& it, unsigned char* st, int slot_i, uint64_t* bar, int gc) {
             const int g = it.group();  // the stage's units are blocks g .. g + gc - 1 of tile t
+            if (a_box) {
+                // (always the whole box: chunks past the stage's units are not read, chunks past K are zero)
+                if (lane == 0)
+                    asm volatile(
+                        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                        ::"r"(a_slot0 + (uint32_t)slot_i * a_step), "l"(&tmap_a), "r"(0), "r"(m0), "r"(2 * g), "r"(smem_u32(bar))
+                        : "memory");
+                return;
+            }
             for (int m = lane; m < rows; m += 32) {
                 bulk_g2s(st + kStageA + m * kDecARowBytes, p.A + (size_t)(m0 + m) * p.K + (size_t)g * kGroup,
                          (uint32_t)(gc * kGroup * 2), bar);
             }
         };
+        auto rows_tx = [&](int gc) -> uint32_t { return a_box ? kABoxBytes : (uint32_t)(rows * gc * (kGroup * 2)); };
+        if (a_box && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         // 1. packed weights of the first ring-full of stages: they do not depend on the previous kernel
         {
             DecStageIter pre(p);
@@ -306,25 +335,25 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             const int gc = it.units();
             unsigned char* st = stage0 + (size_t)slot * stage_bytes;
             if (n < p.prefetch) {
-                if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)(rows * gc * (kGroup * 2)));
+                if (lane == 0) mbar_expect_tx(&full[slot], rows_tx(gc));
                 __syncwarp();
-                issue_rows(it, st, &full[slot], gc);
+                issue_rows(it, st, slot, &full[slot], gc);
             } else if (n < stages) {
                 // first use of this slot, weights not requested yet: nothing to wait for; the (small) row
                 // copies go in front of the weights
-                if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)gc * unit_tx + (uint32_t)(rows * gc * (kGroup * 2)));
+                if (lane == 0) mbar_expect_tx(&full[slot], (uint32_t)gc * unit_tx + rows_tx(gc));
                 __syncwarp();
-                issue_rows(it, st, &full[slot], gc);
+                issue_rows(it, st, slot, &full[slot], gc);
                 __syncwarp();
                 if (lane == 0) issue_weights(it, st, &full[slot], gc);
             } else {
                 if (!mbar_wait_producer(&empty[slot], phase ^ 1u)) return;  // status recorded
                 if (lane == 0) {
-                    mbar_expect_tx(&full[slot], (uint32_t)gc * unit_tx + (uint32_t)(rows * gc * (kGroup * 2)));
+                    mbar_expect_tx(&full[slot], (uint32_t)gc * unit_tx + rows_tx(gc));
                     issue_weights(it, st, &full[slot], gc);
                 }
                 __syncwarp();
-                issue_rows(it, st, &full[slot], gc);
+                issue_rows(it, st, slot, &full[slot], gc);
             }
             if (++slot == stages) {
                 slot = 0;
@@ -355,8 +384,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
     const uint32_t w_off = (uint32_t)(us * kBlockBytes + hh * 1024 + (tig >> 1) * 128 + ((gq + 4 * (tig >> 1)) & 7) * 16 + (tig & 1) * 8);
     // (a stage holds only the `rows` batch rows this CTA has: lanes of absent rows read the last present one,
     // and what they compute lands in output columns that are never stored)
-    const uint32_t a_off = (uint32_t)(kStageA + us * (kGroup * 2) + min(gq, rows - 1) * kDecARowBytes + tig * 32);
-    const uint32_t a_off1 = (uint32_t)(kStageA + us * (kGroup * 2) + min(8 + gq, rows - 1) * kDecARowBytes + tig * 32);
+    // -- relative to the slot's activation rows; the 64 k of the unit's second half lie kADc further.
+    // Tensor-copy layout: [chunk of 64 k][row][128 B], the 16-byte pieces of a row exchanged by the 128-byte
+    // swizzle (piece j of row r at j ^ (r & 7)): the lane's second 16 bytes are at its first address ^ 16.
+    const int piece = (2 * tig) ^ gq;
+    const uint32_t a_off = a_box ? (uint32_t)(us * 2 * (kRows * 128) + gq * 128 + piece * 16)
+                                 : (uint32_t)(us * (kGroup * 2) + min(gq, rows - 1) * kDecARowBytes + tig * 32);
+    const uint32_t a_off1 = a_box ? a_off + 1024u
+                                  : (uint32_t)(us * (kGroup * 2) + min(8 + gq, rows - 1) * kDecARowBytes + tig * 32);
+    constexpr int kADc = a_box ? kRows * 128 : 128;
     // SG = 4 (groups of 32 k): the lane's 16 k of a 64-k half lie in row 2 c + tig / 2
     const int jlane = SG == 4 ? (tig >> 1) : 0;
     const uint32_t s_off = (uint32_t)(kDecStageS + (us * SG + jlane) * (kSBlockHalves * 2) + (32 * hh + 4 * gq) * 2);
@@ -411,6 +447,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
     int slot = 0;
     uint32_t phase = 0;
     uint32_t st_addr = stage0_addr;
+    uint32_t sa_addr = a_slot0;
     for (int ci = blockIdx.x; ci < p.nchunks; ci += gridDim.x) {
         const int u0 = chunk_begin(p, ci);
         const int u1 = chunk_begin(p, ci + 1);
@@ -423,7 +460,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             const int gc = min(kDecUnitsPerStage, min(u1, tile_end) - u);
             if (!mbar_wait(&full[slot], phase)) return;  // status recorded; every consumer warp sees it
             if (us < gc) {
-                const uint32_t wa = st_addr + w_off, aa = st_addr + a_off, aa1 = st_addr + a_off1;
+                const uint32_t wa = st_addr + w_off, aa = sa_addr + a_off, aa1 = sa_addr + a_off1;
                 if constexpr (SG == 1) load_consts(st_addr, 0);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
@@ -435,7 +472,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
                     for (int mb = 0; mb < MB; ++mb) {
                         uint4 x, y;
                         const uint32_t ab = mb == 0 ? aa : aa1;
-                        if (c == 0) {
+                        if constexpr (a_box) {
+                            if (c == 0) {
+                                x = lds128<0>(ab);
+                                y = lds128<0>(ab ^ 16u);
+                            } else {
+                                x = lds128<kADc>(ab);
+                                y = lds128<kADc>(ab ^ 16u);
+                            }
+                        } else if (c == 0) {
                             x = lds128<0>(ab);
                             y = lds128<16>(ab);
                         } else {
@@ -472,10 +517,12 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const Decod
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[slot]);
             st_addr += (uint32_t)stage_bytes;
+            sa_addr += a_step;
             if (++slot == stages) {
                 slot = 0;
                 phase ^= 1u;
                 st_addr = stage0_addr;
+                sa_addr = a_slot0;
             }
             u += gc;
             if (u != tile_end && u != u1) continue;

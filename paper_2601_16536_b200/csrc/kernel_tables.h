@@ -7,12 +7,13 @@
 
 namespace w4a16 {
 
-typedef void (*DecodeKernel)(const DecodeParams);
+typedef void (*DecodeKernel)(const CUtensorMap, const DecodeParams);
 typedef void (*TileKernel)(const CUtensorMap, const TileParams);
 
 // sg = scale rows per 128-k block (1, 2, 4)
-DecodeKernel decode_kernel_f16(int mb, bool cluster, int sg, bool sym);
-DecodeKernel decode_kernel_bf16(int mb, bool cluster, int sg, bool sym);
+// a_box: activation rows of a stage as one tensor copy
+DecodeKernel decode_kernel_f16(int mb, bool cluster, int sg, bool sym, bool a_box);
+DecodeKernel decode_kernel_bf16(int mb, bool cluster, int sg, bool sym, bool a_box);
 TileKernel tile_kernel_f16_sg1(int mt_index, bool sym, bool epi);
 TileKernel tile_kernel_f16_sg2(int mt_index, bool sym, bool epi);
 TileKernel tile_kernel_f16_sg4(int mt_index, bool sym, bool epi);
