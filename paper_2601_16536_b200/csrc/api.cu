@@ -750,6 +750,7 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     p.stages = g.stages;
     p.stage_bytes = g.stage_bytes;
     p.prefetch = g.prefetch;
+    decode_fill_chunk_math(p);
     p.epi = epi;
     CUtensorMap tmap_a;
     if (g.a_box) {
@@ -898,6 +899,7 @@ int w4a16_gemm_static_ws(const uint16_t* A, const void* Wq, const void* S, const
     p.stages = g.stages;
     p.stage_bytes = g.stage_bytes;
     p.prefetch = g.prefetch;
+    decode_fill_chunk_math(p);
     CUtensorMap tmap_a;
     if (g.a_box) {
         if (!make_decode_tensor_map(&tmap_a, A, M, K, g.mb)) return W4A16_ERR_CUDA;

@@ -49,6 +49,25 @@ __host__ __device__ constexpr int dec_unit_bytes(int sg, bool sym) {
     return kBlockBytes + sg * kSBlockHalves * 2 + (sym ? 0 : sg * kZBlockWords * 4);
 }
 
+// n / d for 0 <= n < 2^31 as a multiplication and a shift: the chunk arithmetic below stands at the head of
+// every CTA's critical path (the producer warp cannot request anything before it knows its first unit), and
+// a hardware-less 32-bit division costs about 100 clocks of dependent instructions, a 64-bit one several
+// hundred.  shift = 31 + ceil(log2 d), mul = ceil(2^shift / d) < 2^32 gives the exact quotient.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+inline FastDiv fast_div_make(uint32_t d) {
+    uint32_t c = 0;
+    while ((1ull << c) < d) ++c;
+    FastDiv f;
+    f.shift = 31 + c;
+    f.mul = (uint32_t)(((1ull << f.shift) + d - 1) / d);
+    return f;
+}
+__device__ __forceinline__ int fast_div(int n, FastDiv f) {
+    return (int)(((unsigned long long)(uint32_t)n * f.mul) >> f.shift);
+}
+
 struct DecodeParams {
     const uint16_t* A;
     const uint32_t* Wq;
@@ -63,8 +82,23 @@ struct DecodeParams {
     int stages;
     int stage_bytes;    // ring stride: decode_stage_bytes(rows of a batch chunk, sg)
     int prefetch;       // stages whose weights are requested before the wait for the previous kernel
+    // chunk arithmetic, prepared by the host (decode_fill_chunk_math)
+    FastDiv div_G, div_split, div_nchunks;
+    int slice_base, slice_rem;   // classic: G / split_k, G % split_k
+    int bal_q, bal_r;            // balanced: (T G) / nchunks, (T G) % nchunks
     Epilogue epi;
 };
+
+inline void decode_fill_chunk_math(DecodeParams& p) {
+    p.div_G = fast_div_make((uint32_t)p.G);
+    p.div_split = fast_div_make((uint32_t)(p.split_k > 0 ? p.split_k : 1));
+    p.div_nchunks = fast_div_make((uint32_t)p.nchunks);
+    p.slice_base = p.split_k > 0 ? p.G / p.split_k : 0;
+    p.slice_rem = p.split_k > 0 ? p.G % p.split_k : 0;
+    const long long units = (long long)p.T * p.G;
+    p.bal_q = (int)(units / p.nchunks);
+    p.bal_r = (int)(units % p.nchunks);
+}
 
 // Activation rows of a stage, two ways (template parameter ABOX of the kernel).  Few rows: one bulk copy per row into the tail of the weight stage
 // (1 KiB + 16 B apart).  More rows: every bulk copy costs the producer warp about 50 clocks whatever its
@@ -184,10 +218,10 @@ __device__ __forceinline__ bool mbar_wait_producer(uint64_t* bar, uint32_t parit
 
 // First unit of chunk i (i == nchunks gives the end of the last chunk).
 __device__ __forceinline__ int chunk_begin(const DecodeParams& p, int i) {
-    if (p.split_k == 0) return (int)(((long long)i * ((long long)p.T * p.G)) / p.nchunks);
-    const int t = i / p.split_k, s = i - t * p.split_k;
-    const int base = p.G / p.split_k, rem = p.G % p.split_k;
-    return t * p.G + s * base + min(s, rem);
+    // balanced: floor(i (T G) / nchunks) = i q + floor(i r / nchunks) with T G = q nchunks + r  (i r < nchunks^2)
+    if (p.split_k == 0) return i * p.bal_q + fast_div(i * p.bal_r, p.div_nchunks);
+    const int t = fast_div(i, p.div_split), s = i - t * p.split_k;
+    return t * p.G + s * p.slice_base + min(s, p.slice_rem);
 }
 // The chunk that holds unit u.
 __device__ __forceinline__ int chunk_of(const DecodeParams& p, int u) {
@@ -213,7 +247,7 @@ struct DecStageIter {
             if (u < u1) break;
             ci += (int)gridDim.x;
         }
-        t = u / p.G;
+        t = fast_div(u, p.div_G);
         tile_end = (t + 1) * p.G;
     }
     __device__ __forceinline__ bool valid() const { return ci < p.nchunks; }
@@ -275,14 +309,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __gri
     // (Batch rows this CTA does not have are never loaded: an MMA column only feeds its own output
     // column, and those columns are not stored.)
     __syncthreads();
-    // CL: every CTA of the cluster is running and has initialised its barriers before anyone writes to
-    // another CTA's shared memory.  All threads of all CTAs of the cluster pass here unconditionally
-    // (the hardware launches a cluster's CTAs together); every later wait in this kernel is a bounded
+    // CL: every CTA of the cluster must be running and have initialised its barriers before anyone writes to
+    // another CTA's shared memory.  All threads of all CTAs of the cluster arrive here unconditionally (the
+    // hardware launches a cluster's CTAs together), so the matching wait cannot hang; it stands where the
+    // guarantee is needed, in front of the exchange (the barrier takes half a microsecond to complete, and
+    // the producer warp has requests to make meanwhile).  Every other wait in this kernel is a bounded
     // mbarrier wait.
-    if (CL) {
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    }
+    // (relaxed: the barrier initialisations were published by fence_mbar_init above, and a releasing arrival
+    // costs the 800 clocks of a cluster-wide memory fence)
+    if (CL) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
     // Let the next kernel in the stream start its own prologue and weight prefetch; everything below
     // that reads or writes memory another kernel may have written comes after griddepcontrol.wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -315,8 +350,9 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __gri
         auto rows_tx = [&](int gc) -> uint32_t { return a_box ? kABoxBytes : (uint32_t)(rows * gc * (kGroup * 2)); };
         if (a_box && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         // 1. packed weights of the first ring-full of stages: they do not depend on the previous kernel
+        const DecStageIter first(p);
         {
-            DecStageIter pre(p);
+            DecStageIter pre(first);
             for (int i = 0; i < p.prefetch && pre.valid(); ++i, pre.next()) {
                 if (lane == 0) {
                     const int gc = pre.units();
@@ -331,7 +367,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __gri
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int slot = 0, n = 0;
         uint32_t phase = 0;
-        for (DecStageIter it(p); it.valid(); it.next(), ++n) {
+        for (DecStageIter it(first); it.valid(); it.next(), ++n) {
             const int gc = it.units();
             unsigned char* st = stage0 + (size_t)slot * stage_bytes;
             if (n < p.prefetch) {
@@ -360,6 +396,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __gri
                 phase ^= 1u;
             }
         }
+        if (CL) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // (pairs with the arrival)
         return;
     }
 
@@ -453,7 +490,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __gri
         const int u1 = chunk_begin(p, ci + 1);
         if (u0 >= u1) continue;
         int u = u0;
-        int t = u / p.G;
+        int t = fast_div(u, p.div_G);
         int tile_end = (t + 1) * p.G;
         int seg_start = u0;
         while (u < u1) {
@@ -548,6 +585,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) gemm_decode_kernel(const __gri
             if (CL && !whole) {
                 // slices 1 .. S - 1 -> slot rank - 1 of the exchange buffer of the cluster's CTA 0, which
                 // adds them to its own slice 0 in ascending order
+                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // the arrival at kernel start
                 uint32_t rank;
                 asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
                 if (rank != 0) {
