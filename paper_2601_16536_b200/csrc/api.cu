@@ -684,6 +684,8 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
             if (g.tiles > kTileMaxTicketTiles) return W4A16_ERR_SPLITK;
             if (ws_body_bytes < tile_workspace_bytes(g)) return W4A16_ERR_WORKSPACE;
         }
+        // (the kernel's chunk arithmetic is 32-bit)
+        if ((long long)g.tiles * G >= (1ll << 31)) return W4A16_ERR_SHAPE;
         CUtensorMap tmap;
         if (!make_act_tensor_map(&tmap, A, M, K, g.mt)) return W4A16_ERR_CUDA;
         TileParams p;
@@ -699,6 +701,7 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         p.split_k = g.split_k;
         p.nchunks = g.nchunks;
         p.stages = g.stages;
+        tile_fill_chunk_math(p);
         p.epi = epi;
         const bool has_epi = bias != nullptr || act != W4A16_ACT_NONE;
         TileKernel kern = tile_kernel(g.mt_index, sg, bf, sym, has_epi);

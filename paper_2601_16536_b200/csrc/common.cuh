@@ -184,6 +184,25 @@ __device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gmem_src, u
         : "memory");
 }
 
+// n / d for 0 <= n < 2^31 as a multiplication and a shift: the chunk arithmetic of the kernels stands at the head of
+// every CTA's critical path (the producer warp cannot request anything before it knows its first unit), and
+// a hardware-less 32-bit division costs about 100 clocks of dependent instructions, a 64-bit one several
+// hundred.  shift = 31 + ceil(log2 d), mul = ceil(2^shift / d) < 2^32 gives the exact quotient.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+inline FastDiv fast_div_make(uint32_t d) {
+    uint32_t c = 0;
+    while ((1ull << c) < d) ++c;
+    FastDiv f;
+    f.shift = 31 + c;
+    f.mul = (uint32_t)(((1ull << f.shift) + d - 1) / d);
+    return f;
+}
+__device__ __forceinline__ int fast_div(int n, FastDiv f) {
+    return (int)(((unsigned long long)(uint32_t)n * f.mul) >> f.shift);
+}
+
 // Tiled tensor copies (TMA) global -> shared; completion as transaction bytes on an mbarrier.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(

@@ -101,8 +101,24 @@ struct TileParams {
     int split_k;     // 0: balanced chunks; S >= 1: classic Split-K
     int nchunks;
     int stages;
+    // chunk arithmetic, prepared by the host (tile_fill_chunk_math); units = m_tiles n_tiles G < 2^31
+    FastDiv div_G, div_split, div_nchunks, div_ntiles;
+    int slice_base, slice_rem;   // classic: G / split_k, G % split_k
+    int bal_q, bal_r;            // balanced: units / nchunks, units % nchunks
     Epilogue epi;
 };
+
+inline void tile_fill_chunk_math(TileParams& p) {
+    p.div_G = fast_div_make((uint32_t)p.G);
+    p.div_split = fast_div_make((uint32_t)(p.split_k > 0 ? p.split_k : 1));
+    p.div_nchunks = fast_div_make((uint32_t)p.nchunks);
+    p.div_ntiles = fast_div_make((uint32_t)p.n_tiles);
+    p.slice_base = p.split_k > 0 ? p.G / p.split_k : 0;
+    p.slice_rem = p.split_k > 0 ? p.G % p.split_k : 0;
+    const long long units = (long long)p.m_tiles * p.n_tiles * p.G;
+    p.bal_q = (int)(units / p.nchunks);
+    p.bal_r = (int)(units % p.nchunks);
+}
 
 // ------------------------------------------------------------------ tcgen05 / TMA wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -195,21 +211,17 @@ __host__ __device__ constexpr uint32_t tile_idesc(int mt, bool bf) {
 }
 
 // ------------------------------------------------------------------ chunk schedule
-// (The out-of-line functions below take the schedule in scalars: registers, not a reference to the kernel's
-// parameter block, which would be copied to local memory for every call.)
-// First unit of chunk i (i == nchunks gives the end of the last chunk).  (64-bit divisions: these two and
-// tile_chunk_start below are functions of their own, called once per chunk -- inlined into every role's
-// walk they made up three quarters of the kernel's code, more than the instruction cache holds.)
-static __device__ __noinline__ long long tile_chunk_begin_s(int split_k, int G, int nchunks, long long units, int i) {
-    if (split_k == 0) return ((long long)i * units) / nchunks;
-    const int t = i / split_k, s = i - t * split_k;
-    const int base = G / split_k, rem = G % split_k;
-    return (long long)t * G + s * base + min(s, rem);
+// First unit of chunk i (i == nchunks gives the end of the last chunk).  Multiply-and-shift divisions with the
+// host's constants: every role's walk starts here, ahead of its first request, and with real divisions (two of
+// them 64-bit) this was the larger part of the kernel's code and a good microsecond of every launch.
+__device__ __forceinline__ int tile_chunk_begin(const TileParams& p, int i) {
+    // balanced: floor(i units / nchunks) = i q + floor(i r / nchunks), units = q nchunks + r  (i r < nchunks^2)
+    if (p.split_k == 0) return i * p.bal_q + fast_div(i * p.bal_r, p.div_nchunks);
+    const int t = fast_div(i, p.div_split), s = i - t * p.split_k;
+    return t * p.G + s * p.slice_base + min(s, p.slice_rem);
 }
-__device__ __forceinline__ long long tile_chunk_begin(const TileParams& p, int i) {
-    return tile_chunk_begin_s(p.split_k, p.G, p.nchunks, (long long)p.m_tiles * p.n_tiles * p.G, i);
-}
-// The chunk that holds unit u.
+// The chunk that holds unit u.  (Out of line and with scalar arguments -- a reference to the kernel's parameter
+// block would be copied to local memory for every call; only the Split-K epilogue of balanced chunks comes here.)
 static __device__ __noinline__ int tile_chunk_of_s(int split_k, int G, int nchunks, long long units, long long u) {
     if (split_k == 0) return (int)(((u + 1) * nchunks - 1) / units);
     const int t = (int)(u / G), g = (int)(u - (long long)t * G);
@@ -229,23 +241,21 @@ struct ChunkStart {
     int g0;        // first group inside the tile
     int len;       // units of the chunk
 };
-static __device__ __noinline__ ChunkStart tile_chunk_start(int split_k, int G, int nchunks, int n_tiles, long long units,
-                                                           int ci, int stride) {
+__device__ __forceinline__ ChunkStart tile_chunk_start(const TileParams& p, int ci, int stride) {
     ChunkStart c;
-    long long u0 = 0;
-    int len = 0;
-    while (ci < nchunks) {
-        u0 = tile_chunk_begin_s(split_k, G, nchunks, units, ci);
-        len = (int)(tile_chunk_begin_s(split_k, G, nchunks, units, ci + 1) - u0);
+    int u0 = 0, len = 0;
+    while (ci < p.nchunks) {
+        u0 = tile_chunk_begin(p, ci);
+        len = tile_chunk_begin(p, ci + 1) - u0;
         if (len > 0) break;
         ci += stride;
     }
     c.ci = ci;
     c.len = len;
-    c.t = (int)(u0 / G);
-    c.g0 = (int)(u0 - (long long)c.t * G);
-    c.mt_i = c.t / n_tiles;
-    c.nt = c.t - c.mt_i * n_tiles;
+    c.t = fast_div(u0, p.div_G);
+    c.g0 = u0 - c.t * p.G;
+    c.mt_i = fast_div(c.t, p.div_ntiles);
+    c.nt = c.t - c.mt_i * p.n_tiles;
     return c;
 }
 
@@ -253,7 +263,7 @@ static __device__ __noinline__ ChunkStart tile_chunk_start(int split_k, int G, i
 // tile).  Every role of the CTA runs its own copy and sees the same sequence.  A warp runs dependent
 // scalar code at only one instruction every several clocks, and the producer and MMA warps sit on
 // the critical path of every stage: so all per-stage work of the roles is a plain counted loop over
-// the segment's 2 * units stages, and the divisions and 64-bit arithmetic happen here, once per chunk.
+// the segment's 2 * units stages, and the chunk arithmetic happens here, once per chunk.
 struct SegWalk {
     const TileParams& p;
     int ci;            // current chunk
@@ -270,8 +280,7 @@ struct SegWalk {
         load_chunk();
     }
     __device__ __forceinline__ void load_chunk() {
-        const ChunkStart c = tile_chunk_start(p.split_k, p.G, p.nchunks, p.n_tiles, (long long)p.m_tiles * p.n_tiles * p.G, ci,
-                                              (int)gridDim.x);
+        const ChunkStart c = tile_chunk_start(p, ci, (int)gridDim.x);
         ci = c.ci;
         if (ci >= p.nchunks) return;
         t = c.t;
