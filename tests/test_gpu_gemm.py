@@ -160,3 +160,17 @@ def test_cluster_exchange_and_workspace_exchange_give_the_same_bits(M, split_k):
     ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
     assert_close(c_f64(got), ref, "M%d split %d" % (M, split_k))
     del ws
+
+
+# The warp-MMA kernel brings a stage's activation rows either as one bulk copy per row (one batch row, or
+# K < 512) or as one tensor copy of 8 or 16 rows x 512 k (rows past M and k past K read as zero): both
+# forms at every edge -- K below, at and above one box, K not a multiple of the box, M at the block edges.
+@pytest.mark.parametrize("K", [128, 384, 512, 640, 1024])
+@pytest.mark.parametrize("M", [2, 7, 8, 9, 15, 16])
+def test_activation_row_paths(M, K):
+    N = 192
+    d = wl.make_problem(M, K, N, seed=31 * M + K)
+    ref = oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128)
+    for split_k in (0, 1):
+        C = _run(d, M, N, K, split_k, B.PATH_DECODE)
+        assert_close(c_f64(C), ref, "decode M%d K%d S%d" % (M, K, split_k))
