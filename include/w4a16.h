@@ -189,9 +189,12 @@ int w4a16_quantize(const uint16_t *W16, uint32_t *Wq_raw, uint16_t *S_raw, uint8
 /* End-to-end form of w4a16_gemm for callers whose activations live in HOST memory:
  * copies A_host (FP16 [M, K], ideally pinned) into the caller's device staging buffer
  * A_dev, runs w4a16_gemm into the device staging buffer C_dev, and copies the result
- * into C_host (FP16 [M, N]); all three steps are enqueued on `stream` in order.  The
- * host buffers must stay valid until the stream has run them.  Weights stay resident
- * on the device (they are the model's parameters, packed once). */
+ * into C_host (FP16 [M, N]); all three steps are enqueued on `stream` in order.  If
+ * C_host is page-locked host memory that the device can address (cudaHostAlloc /
+ * cudaHostRegister, 16-byte aligned), the kernel stores the result there itself: the
+ * copy is skipped and C_dev is not written.  The host buffers must stay valid until the
+ * stream has run them.  Weights stay resident on the device (they are the model's
+ * parameters, packed once). */
 int w4a16_gemm_host(const uint16_t *A_host, uint16_t *A_dev, const void *Wq, const void *S,
                     const void *Z, uint16_t *C_dev, uint16_t *C_host, int M, int N, int K,
                     int group, int split_k, w4a16_stream_t stream);

@@ -241,8 +241,9 @@ def w4a16_gemm(A: torch.Tensor, pw: PackedWeights, C: Optional[torch.Tensor] = N
 def w4a16_gemm_host(A_host: torch.Tensor, A_dev: torch.Tensor, pw: PackedWeights,
                     C_dev: torch.Tensor, C_host: torch.Tensor, split_k: int = 0,
                     stream: Optional[int] = None) -> None:
-    """Host activations in, host result out (pinned tensors); copies and GEMM on ``stream`` (a raw
-    ``cudaStream_t`` handle, e.g. ``torch.cuda.Stream().cuda_stream``) or, by default, on the current stream."""
+    """Host activations in, host result out; copies and GEMM on ``stream`` (a raw ``cudaStream_t`` handle,
+    e.g. ``torch.cuda.Stream().cuda_stream``) or, by default, on the current stream.  A pinned ``C_host`` is
+    written by the kernel itself and ``C_dev`` is then left untouched; a pageable one goes through ``C_dev``."""
     M = A_host.shape[0]
     _check(load().w4a16_gemm_host(_ptr(A_host), _ptr(A_dev), _ptr(pw.Wq), _ptr(pw.S), _ptr(pw.Z),
                                   _ptr(C_dev), _ptr(C_host), M, pw.N, pw.K, pw.group, split_k,

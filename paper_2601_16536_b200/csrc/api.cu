@@ -839,9 +839,22 @@ int w4a16_gemm_host(const uint16_t* A_host, uint16_t* A_dev, const void* Wq, con
         cudaGetLastError();
         return W4A16_ERR_CUDA;
     }
-    int rc = w4a16_gemm(A_dev, Wq, S, Z, C_dev, M, N, K, group, split_k, stream);
+    // Page-locked host memory that the device can address takes the result straight from the kernel's stores
+    // (each element of C is written once, by whoever finishes its sum): one copy and one runtime call less.
+    // Anything else goes through C_dev and a copy.
+    uint16_t* c_direct = nullptr;
+    {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, C_host) == cudaSuccess) {
+            if (attr.type == cudaMemoryTypeHost && attr.devicePointer != nullptr && aligned16(attr.devicePointer))
+                c_direct = static_cast<uint16_t*>(attr.devicePointer);
+        } else {
+            cudaGetLastError();
+        }
+    }
+    int rc = w4a16_gemm(A_dev, Wq, S, Z, c_direct ? c_direct : C_dev, M, N, K, group, split_k, stream);
     if (rc != W4A16_OK) return rc;
-    if (cudaMemcpyAsync(C_host, C_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    if (!c_direct && cudaMemcpyAsync(C_host, C_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
         cudaGetLastError();
         return W4A16_ERR_CUDA;
     }

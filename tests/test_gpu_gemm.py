@@ -125,19 +125,30 @@ def test_workspace_errors():
     torch.cuda.synchronize()
 
 
-def test_host_buffer_entry_point_matches_device_call():
-    M, K, N = 8, 1024, 256
-    d = wl.make_problem(M, K, N, seed=95)
+# Host result buffer: page-locked memory takes the kernel's stores directly (the device staging buffer is then
+# left alone), ordinary pageable memory gets the result through the staging buffer and a copy.  Both on the
+# warp-MMA kernel (M = 8) and the tcgen05 kernel (M = 40).
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("M", [8, 40])
+def test_host_buffer_entry_point_matches_device_call(M, pinned):
+    K, N = 1024, 256
+    d = wl.make_problem(M, K, N, seed=95 + M)
     pw = pack_problem(d, N, K)
     ws = ensure_ws(M, N, K, 0)
     A_host = torch.from_numpy(d["A"].view(np.float16)).pin_memory()
-    C_host = torch.empty((M, N), dtype=torch.float16).pin_memory()
+    C_host = torch.zeros((M, N), dtype=torch.float16)
+    if pinned:
+        C_host = C_host.pin_memory()
     A_dev = torch.empty((M, K), dtype=torch.float16, device="cuda")
-    C_dev = torch.empty((M, N), dtype=torch.float16, device="cuda")
-    B.w4a16_gemm_host(A_host, A_dev, pw, C_dev, C_host)
-    torch.cuda.synchronize()
+    C_dev = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    for _ in range(2):
+        B.w4a16_gemm_host(A_host, A_dev, pw, C_dev, C_host)
+        torch.cuda.synchronize()
     C = B.w4a16_gemm(to_dev(d["A"]), pw)
     assert np.array_equal(C_host.numpy().view(np.uint16), c_bits(C))
+    if not pinned:
+        assert np.array_equal(c_bits(C_dev), c_bits(C))
+    assert B.w4a16_device_status() == 0
     del ws
 
 
