@@ -397,17 +397,16 @@ bool make_decode_tensor_map(CUtensorMap* map, const void* A, int M, int K, int m
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Path taken when the caller does not force one.  Measured on B200: up to 8 batch rows the warp-MMA
-// kernel is ahead everywhere (K = 11008 / N = 4096: 9.8 us against 12.9; K = 28672 / N = 8192: 34 against
-// 44).  From 9 to 16 rows it needs a second batch block per weight; it still wins where its K slices
-// exchange through a cluster (M = 16: 12.5 against 12.9 us at K = 11008 / N = 4096, 6.9 against 8.6 at
-// K = N = 4096) and loses where they cannot (16.9 against 16.5 at N = 12288, 46.3 against 44.7 at
-// K = 28672 / N = 8192).  Above 16 rows the tcgen05 kernel.
+// Path taken when the caller does not force one.  Measured on B200 (us, warp-MMA kernel / tcgen05 kernel): up to
+// 16 batch rows the warp-MMA kernel is ahead or level everywhere, with or without a cluster exchange (M = 16:
+// K = 11008 / N = 4096 10.8 / 12.2, K = N = 4096 6.0 / 7.9, K = 4096 / N = 12288 12.5 / 13.1, K = 4096 /
+// N = 22016 18.8 / 21.7, K = 28672 / N = 8192 40.6 / 41.2, K = 18432 / N = 7168 26.4 / 26.7); from 17 rows on it
+// needs a second pass over the weights and the tcgen05 kernel wins by 1.4 to 2 times (M = 24: 22.5 / 12.8 and
+// 75.8 / 42.2 on the first and the last of those shapes).
 int resolve_path(int M, int N, int G, int split_k, int sms, int path, bool allow_cluster = true) {
+    (void)N; (void)G; (void)split_k; (void)sms; (void)allow_cluster;
     if (path != W4A16_PATH_AUTO) return path;
-    if (M <= 8) return W4A16_PATH_DECODE;
-    if (M <= 16 && decode_geom(M, N, G, split_k, sms, allow_cluster).cluster) return W4A16_PATH_DECODE;
-    return W4A16_PATH_TILE;
+    return M <= 16 ? W4A16_PATH_DECODE : W4A16_PATH_TILE;
 }
 
 // FP32 partials of the two-kernel reduce used by the plain path: [split_k][M][N].

@@ -106,16 +106,11 @@ def test_path_and_schedule_rules_at_the_benchmark_shapes(lib):
     DECODE, TILE = 2, 3
     path = lambda M, N, K: lib.w4a16_choose_path(M, N, K, 128)
     split = lambda M, N, K: lib.w4a16_choose_split_k(M, N, K, 128)
-    # up to 8 rows: always the warp-MMA kernel
-    for N, K in [(4096, 4096), (4096, 11008), (8192, 28672), (22016, 4096), (1536, 6144)]:
-        for M in (1, 4, 8):
+    # up to 16 rows (one pass of the warp-MMA kernel over the weights): always that kernel
+    for N, K in [(4096, 4096), (4096, 11008), (8192, 28672), (22016, 4096), (1536, 6144), (12288, 4096)]:
+        for M in (1, 4, 8, 9, 16):
             assert path(M, N, K) == DECODE
-    # 9 .. 16 rows: the warp-MMA kernel where its K slices form clusters, else tcgen05
-    assert path(16, 4096, 11008) == DECODE and split(16, 4096, 11008) == 4
-    assert path(16, 4096, 4096) == DECODE
-    assert path(16, 12288, 4096) == TILE
-    assert path(16, 22016, 4096) == TILE
-    assert path(16, 8192, 28672) == TILE
+    assert split(16, 4096, 11008) == 4
     # above 16 rows: tcgen05
     for M in (17, 32, 64, 256, 4096):
         assert path(M, 4096, 11008) == TILE
