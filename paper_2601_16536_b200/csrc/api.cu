@@ -161,8 +161,11 @@ DecodeGeom decode_geom(int M, int N, int G, int split_k, int sms, bool allow_clu
         // 13 (1.3 / 2.8 / about 4 us at 0.3 us per unit).  K = 4096 / N = 22016: whole tiles 15.0 us,
         // balanced 18.1; K = 28672 / N = 8192: two slices 33.8, balanced 34.3; K = 11008 / N = 4096:
         // four slices 9.7, three 10.5, two 13.5; K = 6144 / N = 1536: six slices in a cluster 4.8,
-        // twelve through the workspace 6.5.
-        long best = (units + slots - 1) / slots + 13;
+        // twelve through the workspace 6.5.  Equal chunks over every slot also run 8 % longer than their
+        // share of the units says (SMs finish the same work up to 8 % apart, and with every slot taken there
+        // is no slack): K = 28672 / N = 8192 balanced 32.4 / two slices in a cluster 31.7 us at M = 1, 40.6 /
+        // 38.7 at M = 16; K = 22016 / N = 8192 26.6 / 25.1; but K = 8192 / N = 10240 balanced 16.5 / whole 18.7.
+        long best = (units * 27 / 25 + slots - 1) / slots + 13;
         int best_s = 0;
         if (T > slots) {
             // more tiles than CTAs: whole tiles dealt round-robin; the CTAs of an SM share its issue
