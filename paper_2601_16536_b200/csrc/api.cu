@@ -108,12 +108,6 @@ int sm_count_or_default() {
     return 148;
 }
 
-bool cluster_ok_or_default() {
-    DeviceState* d = nullptr;
-    if (current_device(&d) == W4A16_OK) return d->cluster_ok;
-    return true;
-}
-
 // ---- decode-path launch geometry ------------------------------------------------
 int decode_mb(int M) { return M <= 8 ? 1 : 2; }
 
@@ -406,8 +400,7 @@ bool make_decode_tensor_map(CUtensorMap* map, const void* A, int M, int K, int m
 // N = 22016 18.8 / 21.7, K = 28672 / N = 8192 40.6 / 41.2, K = 18432 / N = 7168 26.4 / 26.7); from 17 rows on it
 // needs a second pass over the weights and the tcgen05 kernel wins by 1.4 to 2 times (M = 24: 22.5 / 12.8 and
 // 75.8 / 42.2 on the first and the last of those shapes).
-int resolve_path(int M, int N, int G, int split_k, int sms, int path, bool allow_cluster = true) {
-    (void)N; (void)G; (void)split_k; (void)sms; (void)allow_cluster;
+int resolve_path(int M, int path) {
     if (path != W4A16_PATH_AUTO) return path;
     return M <= 16 ? W4A16_PATH_DECODE : W4A16_PATH_TILE;
 }
@@ -466,7 +459,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return 1;
     int G = K / kGroup;
-    switch (resolve_path(M, N, G, 0, sm_count_or_default(), path, cluster_ok_or_default())) {
+    switch (resolve_path(M, path)) {
         case W4A16_PATH_DECODE: return choose_split_decode(M, N, G, sm_count_or_default());
         case W4A16_PATH_TILE: return choose_split_tile(M, N, G, sm_count_or_default());
         default: return 1;
@@ -475,7 +468,7 @@ int w4a16_choose_split_k_ex(int M, int N, int K, int group, int path) {
 int w4a16_choose_path(int M, int N, int K, int group) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (check_weight_shape(N, K, group) != W4A16_OK || M < 1) return W4A16_ERR_SHAPE;
-    return resolve_path(M, N, K / kGroup, 0, sm_count_or_default(), W4A16_PATH_AUTO, cluster_ok_or_default());
+    return resolve_path(M, W4A16_PATH_AUTO);
 }
 int w4a16_choose_split_k(int M, int N, int K, int group) {
     return w4a16_choose_split_k_ex(M, N, K, group, W4A16_PATH_AUTO);
@@ -642,7 +635,7 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
     if (!d->is_sm100) return W4A16_ERR_ARCH;
 
     const int path_asked = path;
-    path = resolve_path(M, N, G, split_k, d->sm_count, path, d->cluster_ok);
+    path = resolve_path(M, path);
     if (split_k > 65535) return W4A16_ERR_SPLITK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t* Zw = sym ? nullptr : static_cast<const uint32_t*>(Z);
