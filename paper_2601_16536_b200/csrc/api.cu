@@ -698,7 +698,15 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         p.stages = g.stages;
         tile_fill_chunk_math(p);
         p.epi = epi;
-        const bool has_epi = bias != nullptr || act != W4A16_ACT_NONE;
+        // Slices of whole tiles on CTAs of their own: the sum of the partial tiles (and with it the optional
+        // bias / activation) is a second, GPU-wide kernel behind this one (kernels_basic.cuh).  Balanced
+        // chunks, whose pieces belong to different tiles, keep the reduce inside the kernel.
+        // Measured (us, in the kernel / second kernel): M = 256: K = 10240 / N = 4608 (four slices) 31.9 / 24.6,
+        // K = 16384 / N = 4096 39.2 / 32.9, K = N = 8192 (two slices) 34.1 / 33.3; 64-row tiles are level (16.6 /
+        // 16.5 at K = 11008 / N = 4096) and 32-row tiles lose the extra launch (12.9 / 13.7): from 128 rows on.
+        const bool defer = g.split_k >= 2 && g.mt >= 128;
+        p.defer_reduce = defer ? 1 : 0;
+        const bool has_epi = !defer && (bias != nullptr || act != W4A16_ACT_NONE);
         TileKernel kern = tile_kernel(g.mt_index, sg, bf, sym, has_epi);
         bool& attr_set = d->tile_attr_set[g.mt_index][log2_sg(sg)][bf ? 1 : 0][sym ? 1 : 0][has_epi ? 1 : 0];
         if (!attr_set) {
@@ -724,6 +732,25 @@ int gemm_locked(const uint16_t* A, const void* Wq, const void* S, const void* Z,
         if (cudaLaunchKernelEx(&cfg, kern, tmap, p) != cudaSuccess) {
             cudaGetLastError();
             return W4A16_ERR_CUDA;
+        }
+        if (defer) {
+            const long long quads = (long long)g.tiles * g.mt * (kTileCols / 4);
+            cudaLaunchConfig_t rcfg = {};
+            rcfg.gridDim = dim3((unsigned)((quads + 255) / 256), 1, 1);
+            rcfg.blockDim = dim3(256, 1, 1);
+            rcfg.stream = st;
+            rcfg.attrs = attr;      // always behind the GEMM kernel just launched on this stream
+            rcfg.numAttrs = 1;
+            const float* parts = p.ws;
+            const int mt_log2 = 4 + g.mt_index;
+            cudaError_t e = bf ? cudaLaunchKernelEx(&rcfg, tile_splitk_reduce_kernel<true>, parts, C, M, N, mt_log2, g.n_tiles,
+                                                    g.split_k, quads, epi)
+                               : cudaLaunchKernelEx(&rcfg, tile_splitk_reduce_kernel<false>, parts, C, M, N, mt_log2, g.n_tiles,
+                                                    g.split_k, quads, epi);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                return W4A16_ERR_CUDA;
+            }
         }
         return W4A16_OK;
     }

@@ -101,6 +101,7 @@ struct TileParams {
     int split_k;     // 0: balanced chunks; S >= 1: classic Split-K
     int nchunks;
     int stages;
+    int defer_reduce;   // 1: partial tiles are only stored; tile_splitk_reduce_kernel sums them (classic slices)
     // chunk arithmetic, prepared by the host (tile_fill_chunk_math); units = m_tiles n_tiles G < 2^31
     FastDiv div_G, div_split, div_nchunks, div_ntiles;
     int slice_base, slice_rem;   // classic: G / split_k, G % split_k
@@ -688,7 +689,7 @@ gemm_tile_kernel(const __grid_constant__ CUtensorMap tmap_a, const TileParams p)
             __syncwarp();
             if (lane == 0) mbar_arrive(&d_empty[dbuf]);
 
-            if (!whole) {
+            if (!whole && p.defer_reduce == 0) {
                 // Split-K reduce (Algorithm 1, Phase 3), per warp region (32 columns n x MT/4 rows m)
                 __threadfence();
                 __syncwarp();

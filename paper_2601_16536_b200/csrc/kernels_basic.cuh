@@ -235,6 +235,52 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ ws, uint16_t* __r
     C[i] = finish<BF>(acc, (int)(i % (size_t)N), epi);
 }
 
+// Algorithm 1, Phase 3 for the tcgen05 kernel when every column tile is cut into `split_k` slices of its own
+// CTAs: that kernel only stores its FP32 partial tiles (slot 2 (T split_k + s) of [batch row in tile][128
+// columns]) and this one, launched behind it, sums them in ascending s, applies the optional bias /
+// activation and rounds once.  A thread takes four neighbouring columns of one batch row.  Inside the GEMM
+// kernel the same sum was a chain of L2 round trips in the one CTA per tile that finished last (5 to 10 us
+// of a 32 us launch at M = 256); here the whole GPU does it at once.
+template <bool BF>
+__global__ void __launch_bounds__(256)
+tile_splitk_reduce_kernel(const float* __restrict__ ws, uint16_t* __restrict__ C, int M, int N, int mt_log2, int n_tiles,
+                          int split_k, long long quads, Epilogue epi) {
+    // the next kernel of the stream may start its prologue; the partial tiles are the previous kernel's output
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= quads) return;
+    const int mt = 1 << mt_log2;
+    const int nq = (int)(q & 31);                       // which four of the tile's 128 columns
+    const long long r = q >> 5;
+    const int m_local = (int)(r & (mt - 1));
+    const int T = (int)(r >> mt_log2);                  // tile = batch tile * n_tiles + column tile
+    const int mt_i = T / n_tiles, nt = T - mt_i * n_tiles;
+    const int m = mt_i * mt + m_local, n = nt * 128 + nq * 4;
+    if (m >= M || n >= N) return;
+    const size_t slot = (size_t)2 * mt * 128;           // floats between the slots of neighbouring slices
+    const float* src = ws + ((size_t)T * split_k) * slot + (size_t)m_local * 128 + nq * 4;
+    float4 acc = __ldcg(reinterpret_cast<const float4*>(src));
+    int s = 1;
+    for (; s + 3 < split_k; s += 4) {                   // four slices' loads in flight, added in order
+        const float4 x0 = __ldcg(reinterpret_cast<const float4*>(src + (size_t)s * slot));
+        const float4 x1 = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(s + 1) * slot));
+        const float4 x2 = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(s + 2) * slot));
+        const float4 x3 = __ldcg(reinterpret_cast<const float4*>(src + (size_t)(s + 3) * slot));
+        acc.x += x0.x; acc.y += x0.y; acc.z += x0.z; acc.w += x0.w;
+        acc.x += x1.x; acc.y += x1.y; acc.z += x1.z; acc.w += x1.w;
+        acc.x += x2.x; acc.y += x2.y; acc.z += x2.z; acc.w += x2.w;
+        acc.x += x3.x; acc.y += x3.y; acc.z += x3.z; acc.w += x3.w;
+    }
+    for (; s < split_k; ++s) {
+        const float4 x = __ldcg(reinterpret_cast<const float4*>(src + (size_t)s * slot));
+        acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+    }
+    const uint32_t lo = (uint32_t)finish<BF>(acc.x, n, epi) | ((uint32_t)finish<BF>(acc.y, n + 1, epi) << 16);
+    const uint32_t hi = (uint32_t)finish<BF>(acc.z, n + 2, epi) | ((uint32_t)finish<BF>(acc.w, n + 3, epi) << 16);
+    *reinterpret_cast<uint2*>(C + (size_t)m * N + n) = make_uint2(lo, hi);
+}
+
 // Diagnostic: one warp waits on a barrier that nobody ever arrives on, with a limit of `limit_ns`.  The wait
 // runs out, records kStatusMbarTimeout in the status word and the kernel returns normally: the same exit
 // every GEMM kernel takes when one of its waits gives up, exercised without any fault.
