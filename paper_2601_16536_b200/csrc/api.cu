@@ -247,20 +247,23 @@ constexpr size_t kWsFullHeaderBytes = kWsHeaderBytes + kTileTicketBytes;
 constexpr long kTileMaxTicketTiles = kTileTicketBytes / (sizeof(int) * kTileDequantWarps);
 
 // Batch rows per CTA tile: the smallest of 16 .. 256 that covers M -- except that a narrow weight
-// matrix gives such tiles too few of them for 148 SMs (N = 1536 and M = 256: twelve), and the
-// twelve-way Split-K that follows costs more than converting the weights once per narrower batch tile.
-// With 24 tiles or fewer, take the widest narrower tile that gives at least 24 (never 128 rows, which
-// measured slower than 64 everywhere it was tried).  Measured: M = 256, K = 6144 / N = 1536: 42.5 us
-// with 256-row tiles, 14.8 with 64 (torch FP16 matmul 16.7); M = 256, K = 8192 / N = 2048: 38.3 against
-// 19.9; M = 64, N = 1536: 14.5 against 10.1 with 32 rows; M = 32: 10.7 against 9.0 with 16.  From N = 4096
-// on (32 column tiles) the covering tile wins (M = 256, K = 16384: 41.8 against 52.4 us).
+// matrix gives such tiles too few of them for 148 SMs (N = 1536 and M = 64: twelve), and where the Split-K
+// sum is made inside the kernel a twelve-way split costs more than converting the weights once per narrower
+// batch tile: M = 64, N = 1536: 14.5 us with 64-row tiles, 10.1 with 32; M = 32: 10.7 against 9.0 with 16.
+// With 24 tiles or fewer, take the widest narrower tile that gives at least 24.  Tiles of 128 and 256 rows
+// hand that sum to a second kernel, so from twelve column tiles on they stay (us with 64- / 128- / 256-row
+// tiles: M = 256: K = 8192 / N = 2048 19.1 / 17.1 / 16.1, K = 10240 / N = 2048 21.9 / 19.4 / 17.0, K = 8192 /
+// N = 3072 26.8 / 20.9 / 18.6; M = 512, K = 6144 / N = 1536 23.1 / 17.6 / 16.5; M = 128: K = 8192 / N = 2048
+// 13.6 / 13.3 / 15.1, K = 6144 / N = 1536 12.2 / 11.8 / 13.3); with eight column tiles the narrow tile is still
+// ahead (M = 256, K = 4096 / N = 1024: 10.6 / 11.0 / 12.6).
 int tile_mt_index(int M, int N) {
     const int idx = M <= 16 ? 0 : M <= 32 ? 1 : M <= 64 ? 2 : M <= 128 ? 3 : 4;
     const long n_tiles = (N + kTileCols - 1) / kTileCols;
     auto tiles = [&](int i) { return (long)((M + (16 << i) - 1) / (16 << i)) * n_tiles; };
     if (tiles(idx) > 24) return idx;
+    if (idx >= 3 && n_tiles >= 12) return idx;
     for (int i = idx - 1; i >= 0; --i) {
-        if (i == 3) continue;
+        if (i == 3) continue;   // (128 rows were slower than 64 wherever the narrower tile was taken)
         if (tiles(i) >= 24) return i;
     }
     return 0;   // even 16-row tiles are few: take the most there are
