@@ -124,6 +124,34 @@ def test_bias_and_activation_are_applied_before_the_final_rounding(path, M, act)
     del ws
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+def test_bias_and_activation_after_the_second_kernels_sum(bf16):
+    """256-row tiles in K slices: the partial tiles are summed by a kernel of their own, which then also adds
+    the bias and applies the activation before the one rounding."""
+    M, K, N = 150, 1024, 1536
+    d = wl.make_problem(M, K, N, seed=911, bf16=bf16)
+    pw = _pack(d, N, K, 128, False, bf16=bf16)
+    r = np.random.Generator(np.random.PCG64(5))
+    bias32 = r.standard_normal(N).astype(np.float32)
+    if bf16:
+        bias_bits = (bias32.view(np.uint32) >> 16).astype(np.uint16)
+        bias = (bias_bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    else:
+        bias_bits = bias32.astype(np.float16).view(np.uint16)
+        bias = bias_bits.view(np.float16).astype(np.float64)
+    ws = ensure_ws(M, N, K, (0, 4))
+    ref = oracle.epilogue(oracle.gemm(d["A"], d["Wq"], d["S"], d["Z"], M, N, K, 128, bf16=bf16), bias, "silu")
+    for split_k in (0, 4):
+        C = B.w4a16_gemm(_dev16(d["A"], bf16), pw, split_k=split_k, path=B.PATH_TILE, bias=_dev16(bias_bits, bf16), act=B.ACT_SILU)
+        torch.cuda.synchronize()
+        assert B.w4a16_device_status() == 0
+        if bf16:
+            _assert_close_bf16(_f64(C), ref, "bf16 split %d" % split_k)
+        else:
+            assert_close(_f64(C), ref, "f16 split %d" % split_k)
+    del ws
+
+
 # ------------------------------------------------------------------ BF16
 @pytest.mark.parametrize("group,symmetric", [(128, False), (64, False), (32, True)])
 def test_bf16_dequant_is_bit_exact(group, symmetric):

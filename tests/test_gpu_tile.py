@@ -62,6 +62,18 @@ def test_tile_path_exact_inputs_bit_equal_for_every_split():
         assert np.array_equal(c_bits(C), want), "split_k=%d" % split_k
 
 
+def test_wide_batch_tiles_with_slices_bit_equal_for_every_split():
+    # Twelve column tiles keep the 256-row batch tile, and its K slices are summed by the second kernel
+    # (tile_splitk_reduce_kernel) instead of inside the GEMM kernel: same order, so with exact inputs the same
+    # bits as one slice, for a ragged batch (200 of 256 rows) and a ragged slice count (8 groups in 3 slices).
+    M, K, N = 200, 1024, 1536
+    d = wl.make_exact_problem(M, K, N, seed=7250)
+    want = oracle.gemm_int(d["A_int"], d["Wq"], d["E"], d["Z"], M, N, K, 128)
+    for split_k in (1, 0, 2, 3, 4, 8):
+        C = _run(d, M, N, K, split_k)
+        assert np.array_equal(c_bits(C), want), "split_k=%d" % split_k
+
+
 def test_tile_path_bit_identical_run_to_run():
     M, K, N = 96, 4096, 512
     d = wl.make_problem(M, K, N, seed=7300)
