@@ -27,7 +27,9 @@ def _run(d, M, N, K, split_k, path=B.PATH_TILE):
 # tiles, a 64-column tail tile (N = 192, 320), one to many groups
 SHAPES = [(32, 128, 128), (1, 256, 128), (9, 640, 192), (16, 1152, 256), (17, 640, 192), (33, 384, 256), (64, 1152, 128),
           (100, 896, 320), (128, 512, 256), (129, 768, 128), (256, 2048, 384), (300, 1280, 192),
-          (700, 640, 256)]
+          (700, 640, 256),
+          # wide enough (twelve column tiles and more) for the 128- and 256-row batch tiles themselves
+          (120, 512, 1536), (300, 384, 1600)]
 
 
 @pytest.mark.parametrize("M,K,N", SHAPES)
