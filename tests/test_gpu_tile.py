@@ -29,7 +29,9 @@ SHAPES = [(32, 128, 128), (1, 256, 128), (9, 640, 192), (16, 1152, 256), (17, 64
           (100, 896, 320), (128, 512, 256), (129, 768, 128), (256, 2048, 384), (300, 1280, 192),
           (700, 640, 256),
           # wide enough (twelve column tiles and more) for the 128- and 256-row batch tiles themselves
-          (120, 512, 1536), (300, 384, 1600)]
+          (120, 512, 1536), (300, 384, 1600),
+          # wide enough for 64-row batch tiles (more than 24 column tiles), with a 64-column tail tile
+          (64, 640, 3328), (40, 1152, 3392)]
 
 
 @pytest.mark.parametrize("M,K,N", SHAPES)
